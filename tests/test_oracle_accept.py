@@ -1,0 +1,176 @@
+"""Pins for the oracle's speculative acceptance (Eq. 1 and the resampling rule): the losslessness identity
+measured from the oracle's own decisions on a tiny vocabulary (exactly, by locating its decision
+boundaries, and empirically over a million seeded draws), plus special cases.  CPU only."""
+import numpy as np
+from scipy.special import softmax
+
+import oracle
+
+
+def run1(tl, dl, x, ua, ur):
+    n, out, _, _ = oracle.accept(tl[None], dl[None], np.asarray(x, np.int32)[None], np.asarray(ua, np.float32)[None],
+                                 np.asarray([ur], np.float32))
+    return int(n[0]), out[0].tolist()
+
+
+def accept_measure(tl, dl, x):
+    """Lebesgue measure of {u in [0,1): the oracle accepts draft token x at row 0}, by bisection."""
+    if run1(tl, dl, [x], [np.nextafter(np.float32(1), np.float32(0))], 0.5)[0] == 1:
+        return 1.0
+    lo, hi = 0.0, 1.0   # accepted at lo (u=0 accepts whenever P[x] > 0), rejected at hi
+    if run1(tl, dl, [x], [0.0], 0.5)[0] == 0:
+        return 0.0
+    for _ in range(40):
+        mid = np.float32((lo + hi) / 2)
+        if mid == np.float32(lo) or mid == np.float32(hi):
+            break
+        if run1(tl, dl, [x], [mid], 0.5)[0] == 1:
+            lo = float(mid)
+        else:
+            hi = float(mid)
+    return (lo + hi) / 2
+
+
+def resample_measures(tl, dl, x_rej, V, n_grid=4001):
+    """Measure of u_res mapped to each token after a rejection of x_rej: boundaries located by bisection."""
+    def tok(u):
+        n, out = run1(tl, dl, [x_rej], [np.nextafter(np.float32(1), np.float32(0))], u)
+        assert n == 0
+        return out[0]
+    edges, cur, lo = [0.0], tok(0.0), 0.0
+    toks = [cur]
+    while True:
+        # find the first grid point where the token changes, then bisect
+        us = np.linspace(lo, 1.0, n_grid, dtype=np.float64)[1:]
+        nxt = None
+        for u in us:
+            if u < 1.0 and tok(np.float32(u)) != cur:
+                nxt = float(np.float32(u))
+                break
+        if nxt is None:
+            break
+        a, b = lo, nxt
+        for _ in range(40):
+            m = np.float32((a + b) / 2)
+            if m == np.float32(a) or m == np.float32(b):
+                break
+            if tok(m) == cur:
+                a = float(m)
+            else:
+                b = float(m)
+        edges.append((a + b) / 2)
+        cur, lo = tok(np.float32(b)), b
+        toks.append(cur)
+    edges.append(1.0)
+    meas = np.zeros(V)
+    for i, t in enumerate(toks):
+        meas[t] += edges[i + 1] - edges[i]
+    assert toks == sorted(toks)   # inverse CDF in ascending token id
+    return meas
+
+
+def test_lossless_identity_by_enumeration():
+    """sum_x Q[x] * (a_x * [t = x] + (1 - a_x) * r_x[t]) = P[t], with a_x and r_x measured from the oracle."""
+    rng = np.random.default_rng(0)
+    V = 6
+    for trial in range(3):
+        tl = (rng.standard_normal((2, V)) * 1.5).astype(np.float32)
+        dl = (rng.standard_normal((1, V)) * 1.5).astype(np.float32)
+        P = softmax(tl[0].astype(np.float64))
+        Q = softmax(dl[0].astype(np.float64))
+        law = np.zeros(V)
+        acc_total = 0.0
+        for x in range(V):
+            a = accept_measure(tl, dl, x)
+            law[x] += Q[x] * a
+            acc_total += Q[x] * a
+            if a < 1.0:
+                r = resample_measures(tl, dl, x, V)
+                law += Q[x] * (1 - a) * r
+        np.testing.assert_allclose(law, P, atol=3e-6)
+        # per-position acceptance probability = sum min(P, Q) = 1 - TV(P, Q)
+        np.testing.assert_allclose(acc_total, np.minimum(P, Q).sum(), atol=1e-6)
+
+
+def test_lossless_identity_empirical_chain():
+    """A million seeded draws, V = 6, gamma = 3: the token emitted at each reached position follows P_j."""
+    rng = np.random.default_rng(1)
+    V, g, N = 6, 3, 1_000_000
+    tl = (rng.standard_normal((g + 1, V)) * 1.2).astype(np.float32)
+    dl = (tl[:g] + 0.8 * rng.standard_normal((g, V))).astype(np.float32)
+    P, Q = softmax(tl.astype(np.float64), axis=1), softmax(dl.astype(np.float64), axis=1)
+    x = np.stack([rng.choice(V, size=N, p=Q[j]) for j in range(g)], axis=1).astype(np.int32)
+    ua = rng.random((N, g), dtype=np.float32)
+    ur = rng.random(N, dtype=np.float32)
+    n, out, _, _ = oracle.accept(np.broadcast_to(tl, (N, g + 1, V)), np.broadcast_to(dl, (N, g, V)), x, ua, ur)
+    assert n.min() >= 0 and n.max() == g
+    reach = 1.0
+    for j in range(g + 1):
+        sel = n >= j                      # position j was reached (all earlier drafts accepted)
+        cnt = np.bincount(out[sel, j], minlength=V).astype(np.float64)
+        m = sel.sum()
+        np.testing.assert_allclose(m / N, reach, atol=4 * np.sqrt(reach * (1 - reach) / N) + 1e-9)
+        sigma = np.sqrt(P[j] * (1 - P[j]) / m)
+        assert np.all(np.abs(cnt / m - P[j]) <= 4.5 * sigma), (j, cnt / m, P[j])
+        chi2 = ((cnt - m * P[j]) ** 2 / (m * P[j])).sum()
+        assert chi2 < 30.0                # 5 degrees of freedom: P(chi2 > 30) ~ 1.5e-5
+        if j < g:
+            reach *= np.minimum(P[j], Q[j]).sum()
+    # accepted prefix is copied verbatim, the tail is -1
+    for j in range(g):
+        assert np.all(out[n > j, j] == x[n > j, j])
+        assert np.all(out[n < j, j] == -1)
+
+
+def test_special_cases():
+    rng = np.random.default_rng(2)
+    V, g = 8, 4
+    tl = rng.standard_normal((g + 1, V)).astype(np.float32)
+    # p = q: always accepted (u < 1), bonus follows the CDF of P_gamma
+    x = rng.integers(0, V, g)
+    n, out = run1(tl, tl[:g].copy(), x, [0.999999] * g, 0.0)
+    assert n == g and out[:g] == x.tolist() and out[g] == 0
+    Pg = softmax(tl[g].astype(np.float64))
+    c = np.cumsum(Pg)
+    for u in (0.05, 0.3, 0.77, 0.999):
+        n, out = run1(tl, tl[:g].copy(), x, [0.5] * g, u)
+        assert out[g] == int(np.searchsorted(c, np.float64(np.float32(u)) * c[-1], side="right"))
+    # draft one-hot on a token the target gives ~0: rejected at row 0, resample ~ P_0 restricted to t != x
+    dl = np.full((g, V), -200.0, np.float32)
+    dl[:, 3] = 0.0
+    tl2 = tl.copy()
+    tl2[:, 3] = -200.0
+    n, out = run1(tl2, dl, [3] * g, [1e-6] * g, 0.4)
+    assert n == 0 and out[1:] == [-1] * g and out[0] != 3
+    P0 = softmax(tl2[0].astype(np.float64))
+    c = np.cumsum(P0)
+    assert out[0] == int(np.searchsorted(c, np.float64(np.float32(0.4)) * c[-1], side="right"))
+    # u_acc = 0 accepts whenever P[x] > 0
+    dl = (tl[:g] + 3 * rng.standard_normal((g, V))).astype(np.float32)
+    n, _ = run1(tl, dl, x, [0.0] * g, 0.5)
+    assert n == g
+    # mid-chain rejection: rows before it accepted, emitted token never equals a token with P <= Q
+    ua = [0.0, 0.0, 0.99999, 0.0]
+    xs = [0, 1, int(np.argmax(softmax(dl[2].astype(np.float64)) - softmax(tl[2].astype(np.float64)))), 2]
+    n, out = run1(tl, dl, xs, ua, 0.5)
+    assert n == 2 and out[:2] == [0, 1] and out[3:] == [-1, -1]
+    Pn, Qn = softmax(tl[2].astype(np.float64)), softmax(dl[2].astype(np.float64))
+    assert Pn[out[2]] > Qn[out[2]]
+    # gamma = 0: only the bonus token
+    n, out, _, _ = oracle.accept(tl[None, :1], np.zeros((1, 0, V), np.float32), np.zeros((1, 0), np.int32),
+                                 np.zeros((1, 0), np.float32), np.asarray([0.0], np.float32))
+    assert n[0] == 0 and out.shape == (1, 1) and out[0, 0] == 0
+
+
+def test_resample_sweep_reproduces_residual_cdf():
+    rng = np.random.default_rng(4)
+    V = 7
+    tl = rng.standard_normal((2, V)).astype(np.float32)
+    dl = rng.standard_normal((1, V)).astype(np.float32)
+    P, Q = softmax(tl[0].astype(np.float64)), softmax(dl[0].astype(np.float64))
+    x = int(np.argmax(Q - P))
+    w = np.maximum(0.0, P - Q)
+    us = (np.arange(2000) + 0.5) / 2000
+    toks = np.array([run1(tl, dl, [x], [0.9999999], u)[1][0] for u in us])
+    np.testing.assert_allclose(np.bincount(toks, minlength=V) / 2000, w / w.sum(), atol=1.5e-3)
+    assert w[x] == 0 and not np.any(toks == x)

@@ -1,0 +1,188 @@
+/*
+ * hippo.h - C ABI of the B200 (sm_100a) hot path of one HIPPO video speculative-decoding step.
+ *
+ * Five operations, each a hand-written CUDA kernel family:
+ *   hippo_select_tokens     semantic-aware visual-token preservation (Section 4.1, Eq. 3-7 + top-k)
+ *   hippo_gather_kv         one-time pruning of the draft model's KV cache (Limitations (i))
+ *   hippo_draft_attention   draft decode attention over the pruned KV (Section 3.2, drafting phase)
+ *   hippo_verify_attention  target verification attention, gamma+1 query tokens (Section 3.2)
+ *   hippo_accept            lossless speculative acceptance (Section 3.2, Eq. 1 and the resampling rule)
+ *
+ * Conventions
+ *   - Every call returns a hippo_status_t (0 = HIPPO_OK, negative = error).  Arguments are validated on the
+ *     host before anything is enqueued; on an error nothing has been launched.
+ *   - Pointers are DEVICE pointers unless the comment says "host".  The caller owns every buffer, including
+ *     workspaces (size them with the *_workspace_bytes helpers; 256-byte aligned).  The library allocates
+ *     no device memory and keeps no state between calls besides a per-thread error string and cached
+ *     kernel attributes.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*) and the call returns without synchronising.
+ *     Calls on different streams may overlap if they use different workspaces and outputs.
+ *   - Device-side waits are bounded.  If one gives up, the kernel records it in the first word of the
+ *     workspace and exits; hippo_workspace_status() reports it after the stream has drained.
+ *   - dtype: HIPPO_DTYPE_FP32 or HIPPO_DTYPE_BF16 storage; accumulation is fp32 (attention) or fp64
+ *     (selection scores, acceptance).
+ */
+#ifndef HIPPO_H_
+#define HIPPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HIPPO_VERSION 100
+#define HIPPO_PAGE_SIZE 64          /* tokens per KV page */
+#define HIPPO_MAX_PACKED_ROWS 128   /* q_len * (n_q_heads / n_kv_heads) must not exceed this */
+
+typedef enum hippo_status {
+    HIPPO_OK = 0,
+    HIPPO_ERR_INVALID_ARG = -1,         /* null pointer, negative size, inconsistent shapes */
+    HIPPO_ERR_UNSUPPORTED_SHAPE = -2,   /* valid in principle, not built (e.g. head_dim not a multiple of 32) */
+    HIPPO_ERR_WORKSPACE_TOO_SMALL = -3,
+    HIPPO_ERR_CUDA = -4,                /* a CUDA runtime/driver call failed; see hippo_last_error() */
+    HIPPO_ERR_TIMEOUT = -5,             /* a bounded device-side wait gave up (reported by hippo_workspace_status) */
+    HIPPO_ERR_UNIMPLEMENTED = -6
+} hippo_status_t;
+
+typedef enum hippo_dtype { HIPPO_DTYPE_FP32 = 0, HIPPO_DTYPE_BF16 = 1 } hippo_dtype_t;
+
+typedef enum hippo_accept_mode { HIPPO_ACCEPT_SAMPLE = 0 } hippo_accept_mode_t;
+
+/* score_mask bits for hippo_select_tokens (Eq. 7 sums the enabled terms) */
+#define HIPPO_SCORE_ATTN 1u
+#define HIPPO_SCORE_TEMP 2u
+#define HIPPO_SCORE_SPA 4u
+#define HIPPO_SCORE_ALL 7u
+
+/*
+ * Paged KV cache of ONE layer.  K and V are separate pools of fixed-size pages:
+ *     k_pages, v_pages : [n_pages][n_kv_heads][HIPPO_PAGE_SIZE][head_dim]   (dtype elements, dense)
+ * so one (page, head) block is a contiguous HIPPO_PAGE_SIZE x head_dim tile.  Token t of sequence b lives in
+ * page  page_table[b * max_pages_per_seq + t / 64]  at slot  t % 64.  A contiguous cache is the special case
+ * page_table == NULL, which means page id = b * max_pages_per_seq + t / 64.  Page ids must lie in
+ * [0, n_pages); slots past a sequence's length may hold anything (they are never used).
+ * Pools must be 128-byte aligned.
+ */
+typedef struct hippo_kv_cache {
+    uint32_t struct_size;        /* sizeof(hippo_kv_cache_t), for versioning */
+    int32_t dtype;               /* hippo_dtype_t */
+    int32_t n_kv_heads;
+    int32_t head_dim;
+    int32_t n_pages;             /* pages in each pool */
+    int32_t max_pages_per_seq;   /* row length of page_table */
+    void *k_pages;
+    void *v_pages;
+    const int32_t *page_table;   /* device int32 [batch][max_pages_per_seq], or NULL for the identity mapping */
+} hippo_kv_cache_t;
+
+/* ---- helpers ------------------------------------------------------------------------------------------------ */
+
+int32_t hippo_version(void);
+const char *hippo_status_string(int32_t status);
+/* Text of the last error raised on the calling host thread (empty string if none). */
+const char *hippo_last_error(void);
+/* Synchronises `stream`, then reads the status word that kernels keep in the first bytes of `workspace`:
+ * HIPPO_OK, or HIPPO_ERR_TIMEOUT if a bounded device-side wait gave up since hippo_workspace_reset(). */
+int32_t hippo_workspace_status(const void *workspace, void *stream);
+/* Zeroes the header of a workspace (status word and arrival counters); enqueued on `stream`.  Must be called
+ * once on a fresh workspace before its first use by the attention calls, and after a reported time-out. */
+int32_t hippo_workspace_reset(void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- selection: Section 4.1 --------------------------------------------------------------------------------- */
+/*
+ * For each of `batch` sequences scores its visual tokens and keeps the k best.
+ *   Eq. 3-4  s_temp = 1 - mean cosine similarity with the same grid cell in the adjacent frames that contain it
+ *   Eq. 5-6  s_spa  = population variance of the token's row of the crop's cosine-similarity matrix (diagonal 1);
+ *            crops are crop_h x crop_w tiles anchored at the grid origin and clipped at the grid edge
+ *   Eq. 7    fused = z(attn_mass) + z(s_spa) + z(s_temp), z = per-frame standardisation (population sigma;
+ *            a frame with constant score contributes 0); only the terms enabled in score_mask are added
+ *   top-k    over the whole sequence, ordered by (fused as fp32 descending, index ascending)
+ * Layout: tokens are frame-major, row-major inside the grid_h x grid_w grid; a sequence whose length is not a
+ * multiple of grid_h*grid_w has a partial last frame holding the first cells.  Sequences are concatenated:
+ * sequence b starts at token offset sum(n_visual[0..b)).
+ *   n_visual  host int32 [batch], each >= 1          k         host int32 [batch], 0 <= k[b] <= n_visual[b]
+ *   embeds    [sum n_visual][embed_dim] dtype         attn_mass fp32 [sum n_visual]
+ *   kept_idx  out int32 [sum k]: sequence b's indices (relative to its own start, ascending) at offset sum(k[0..b))
+ *   fused_score out fp32 [sum n_visual]
+ * Scores are accumulated in fp64.  embed_dim must be a multiple of 8; crop_h*crop_w <= 32.
+ */
+size_t hippo_select_workspace_bytes(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w,
+                                    int32_t crop_h, int32_t crop_w);
+int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w, int32_t crop_h,
+                            int32_t crop_w, int32_t embed_dim, int32_t dtype, const void *embeds,
+                            const float *attn_mass, const int32_t *k, uint32_t score_mask, int32_t *kept_idx,
+                            float *fused_score, void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- gather: pruning the draft KV cache (Limitations (i); experimental set-up: "remove the corresponding
+ *      video features") --------------------------------------------------------------------------------------- */
+/*
+ * For every layer l < n_layers, sequence b and i in [keep_offsets[b], keep_offsets[b+1]):
+ *     dst token (i - keep_offsets[b]) of sequence b  :=  src token keep_idx[i] of sequence b      (K and V, all heads)
+ * `src` / `dst` describe layer 0; layer l's pools start src_layer_stride_bytes * l (dst_layer_stride_bytes * l)
+ * bytes further on.  Page tables are shared by all layers.  keep_idx holds positions in the source sequence
+ * (the kept visual tokens and every always-kept position such as text), ascending per sequence to preserve
+ * order; the kernel does not require ascending order.  Indices are not range-checked on the device: the
+ * caller guarantees 0 <= keep_idx < source length.  src and dst must not overlap and must agree in dtype,
+ * n_kv_heads and head_dim (head_dim * element size a multiple of 16 bytes).
+ *   keep_idx      int32 [total_keep]          keep_offsets  int32 [batch + 1] (device), keep_offsets[0] = 0
+ *   total_keep    host copy of keep_offsets[batch]
+ */
+int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src, size_t src_layer_stride_bytes,
+                        const hippo_kv_cache_t *dst, size_t dst_layer_stride_bytes, int32_t batch,
+                        const int32_t *keep_idx, const int32_t *keep_offsets, int32_t total_keep, void *stream);
+
+/* ---- attention: Section 3.2 (drafting phase / verification phase) ------------------------------------------ */
+/*
+ * out[b][t][h] = softmax_j( scale * q[b][t][h] . K[b][j][h / G] ) V[b][j][h / G],   G = n_q_heads / n_kv_heads,
+ * over the keys j <= kv_len[b] - q_len + t: the q_len query tokens are the LAST q_len positions of the
+ * kv_len[b]-token context (their own K/V are already in the cache), every earlier key is visible.
+ * hippo_verify_attention is tuned for q_len = gamma + 1 rows against the full-length video cache (one persistent
+ * CTA per SM streaming K/V tiles); hippo_draft_attention for q_len = 1 against the short pruned cache
+ * (many small splits).  Both compute the same function for any q_len >= 1.
+ *   q        [batch][q_len][n_q_heads][head_dim] dtype        out  same shape and dtype as q
+ *   kv_len   int32 [batch] (device), q_len <= kv_len[b] <= max_kv_len;  a sequence with kv_len[b] < q_len is skipped
+ *   max_kv_len  host upper bound used to size the launch; <= max_pages_per_seq * 64
+ *   softmax_scale  0 selects 1/sqrt(head_dim)
+ *   num_splits  0 = automatic
+ *   lse      optional fp32 [batch][q_len][n_q_heads], natural-log sum of exponentials of the scaled logits
+ * bf16 with head_dim 64 or 128 runs on the tensor cores with TMA-staged tiles; fp32 (any head_dim that is a
+ * multiple of 32, <= 256) runs on the CUDA cores.  q_len * G <= HIPPO_MAX_PACKED_ROWS.
+ * The workspace header must have been zeroed once with hippo_workspace_reset().
+ */
+size_t hippo_attention_workspace_bytes(int32_t batch, int32_t q_len, int32_t n_q_heads, int32_t n_kv_heads,
+                                       int32_t head_dim);
+int32_t hippo_verify_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, const void *q,
+                               const hippo_kv_cache_t *kv, const int32_t *kv_len, int32_t max_kv_len,
+                               float softmax_scale, int32_t num_splits, void *out, float *lse, void *workspace,
+                               size_t workspace_bytes, void *stream);
+int32_t hippo_draft_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, const void *q,
+                              const hippo_kv_cache_t *kv, const int32_t *kv_len, int32_t max_kv_len,
+                              float softmax_scale, int32_t num_splits, void *out, float *lse, void *workspace,
+                              size_t workspace_bytes, void *stream);
+
+/* ---- acceptance: Section 3.2, Eq. 1 -------------------------------------------------------------------------- */
+/*
+ * Row alignment: target row j in [0, gamma] and draft row j in [0, gamma) both predict draft token x_{j+1};
+ * target row gamma is the bonus row.  P_j, Q_j = softmax of the logit rows (temperature 1).
+ *   for j = 0 .. gamma-1: accept x_{j+1} iff u_accept[j] * Q_j[x] < P_j[x]   (probability min(1, P/Q), Eq. 1)
+ *   n = number accepted before the first rejection
+ *   n < gamma : emit a token drawn from norm(max(0, P_n - Q_n));   n == gamma : from P_gamma
+ *   the draw is the inverse CDF in ascending token id with u_resample[b]: smallest t with cumsum_t > u * total
+ * Softmax normalisers, probabilities and CDFs are evaluated in fp64.
+ *   target_logits fp32 [batch][gamma+1][vocab]     draft_logits fp32 [batch][gamma][vocab]
+ *   draft_tokens  int32 [batch][gamma] in [0, vocab) u_accept fp32 [batch][gamma]    u_resample fp32 [batch]
+ *   n_accepted    out int32 [batch]                 out_tokens out int32 [batch][gamma+1]: accepted draft tokens,
+ *                                                   then the drawn token, then -1
+ */
+size_t hippo_accept_workspace_bytes(int32_t batch, int32_t gamma, int32_t vocab);
+int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *target_logits,
+                     const float *draft_logits, const int32_t *draft_tokens, const float *u_accept,
+                     const float *u_resample, int32_t mode, int32_t *n_accepted, int32_t *out_tokens,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIPPO_H_ */

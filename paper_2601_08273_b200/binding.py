@@ -1,0 +1,249 @@
+"""Thin ctypes binding of libhippo.so: same names as the C ABI (include/hippo.h), argument marshalling only.
+
+Every step of the hot path runs in the CUDA library; there is no CPU or PyTorch fallback.  Importing this module
+fails loudly if the library has not been built (`python -m paper_2601_08273_b200.build`).  PyTorch is used for
+device memory and streams only: tensors are passed as raw device pointers.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libhippo.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libhippo.so is missing (%s). Build the CUDA extension first: python -m paper_2601_08273_b200.build. "
+        "There is no fallback path." % LIB_PATH)
+
+lib = ctypes.CDLL(LIB_PATH)
+
+HIPPO_OK = 0
+HIPPO_ERR_INVALID_ARG = -1
+HIPPO_ERR_UNSUPPORTED_SHAPE = -2
+HIPPO_ERR_WORKSPACE_TOO_SMALL = -3
+HIPPO_ERR_CUDA = -4
+HIPPO_ERR_TIMEOUT = -5
+HIPPO_ERR_UNIMPLEMENTED = -6
+HIPPO_DTYPE_FP32 = 0
+HIPPO_DTYPE_BF16 = 1
+HIPPO_SCORE_ALL = 7
+PAGE_SIZE = 64
+
+_vp, _i32, _u32, _sz, _f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_float
+
+
+class KVCacheStruct(ctypes.Structure):
+    _fields_ = [("struct_size", _u32), ("dtype", _i32), ("n_kv_heads", _i32), ("head_dim", _i32),
+                ("n_pages", _i32), ("max_pages_per_seq", _i32), ("k_pages", _vp), ("v_pages", _vp),
+                ("page_table", _vp)]
+
+
+_KVP = ctypes.POINTER(KVCacheStruct)
+_I32P = ctypes.POINTER(_i32)
+
+lib.hippo_version.restype = _i32
+lib.hippo_status_string.restype = ctypes.c_char_p
+lib.hippo_status_string.argtypes = [_i32]
+lib.hippo_last_error.restype = ctypes.c_char_p
+lib.hippo_workspace_status.restype = _i32
+lib.hippo_workspace_status.argtypes = [_vp, _vp]
+lib.hippo_workspace_reset.restype = _i32
+lib.hippo_workspace_reset.argtypes = [_vp, _sz, _vp]
+lib.hippo_select_workspace_bytes.restype = _sz
+lib.hippo_select_workspace_bytes.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32]
+lib.hippo_select_tokens.restype = _i32
+lib.hippo_select_tokens.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _I32P, _u32, _vp, _vp,
+                                    _vp, _sz, _vp]
+lib.hippo_gather_kv.restype = _i32
+lib.hippo_gather_kv.argtypes = [_i32, _KVP, _sz, _KVP, _sz, _i32, _vp, _vp, _i32, _vp]
+lib.hippo_attention_workspace_bytes.restype = _sz
+lib.hippo_attention_workspace_bytes.argtypes = [_i32] * 5
+for _name in ("hippo_verify_attention", "hippo_draft_attention"):
+    getattr(lib, _name).restype = _i32
+    getattr(lib, _name).argtypes = [_i32, _i32, _i32, _vp, _KVP, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _sz, _vp]
+lib.hippo_accept_workspace_bytes.restype = _sz
+lib.hippo_accept_workspace_bytes.argtypes = [_i32, _i32, _i32]
+lib.hippo_accept.restype = _i32
+lib.hippo_accept.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp]
+
+
+class HippoError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        msg = lib.hippo_last_error().decode()
+        super().__init__("%s (%d): %s" % (lib.hippo_status_string(status).decode(), status, msg))
+
+
+def _check(status: int) -> None:
+    if status != HIPPO_OK:
+        raise HippoError(status)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return HIPPO_DTYPE_FP32
+    if t.dtype == torch.bfloat16:
+        return HIPPO_DTYPE_BF16
+    raise TypeError("unsupported dtype %s" % t.dtype)
+
+
+def _host_i32(v: Sequence[int]):
+    arr = (_i32 * len(v))(*[int(x) for x in v])
+    return arr
+
+
+def hippo_version() -> int:
+    return int(lib.hippo_version())
+
+
+class KVCache:
+    """Descriptor of one layer's paged cache; keeps the tensors alive.  k_pages, v_pages:
+    [n_pages][n_kv_heads][64][head_dim]; page_table int32 [batch][max_pages_per_seq] or None (identity)."""
+
+    def __init__(self, k_pages: torch.Tensor, v_pages: torch.Tensor, page_table: Optional[torch.Tensor],
+                 max_pages_per_seq: Optional[int] = None):
+        assert k_pages.is_contiguous() and v_pages.is_contiguous() and k_pages.shape == v_pages.shape
+        assert k_pages.dim() == 4 and k_pages.shape[2] == PAGE_SIZE
+        if page_table is not None:
+            assert page_table.dtype == torch.int32 and page_table.is_contiguous() and page_table.dim() == 2
+            max_pages_per_seq = page_table.shape[1]
+        assert max_pages_per_seq is not None
+        self.k_pages, self.v_pages, self.page_table = k_pages, v_pages, page_table
+        self.struct = KVCacheStruct(ctypes.sizeof(KVCacheStruct), _dtype_code(k_pages), k_pages.shape[1],
+                                    k_pages.shape[3], k_pages.shape[0], int(max_pages_per_seq),
+                                    k_pages.data_ptr(), v_pages.data_ptr(),
+                                    None if page_table is None else page_table.data_ptr())
+
+    @property
+    def n_kv_heads(self) -> int:
+        return self.k_pages.shape[1]
+
+    @property
+    def head_dim(self) -> int:
+        return self.k_pages.shape[3]
+
+
+def new_workspace(n_bytes: int, device="cuda") -> torch.Tensor:
+    """Zero-filled, 256-byte aligned byte buffer (a fresh workspace needs its header zeroed once)."""
+    ws = torch.zeros(max(int(n_bytes), 256), dtype=torch.uint8, device=device)
+    assert ws.data_ptr() % 256 == 0
+    return ws
+
+
+def hippo_workspace_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(lib.hippo_workspace_status(_ptr(workspace), _stream(stream)))
+
+
+def hippo_workspace_reset(workspace: torch.Tensor, stream=None) -> None:
+    _check(lib.hippo_workspace_reset(_ptr(workspace), workspace.numel(), _stream(stream)))
+
+
+# ---- selection --------------------------------------------------------------------------------------------------
+
+def hippo_select_workspace_bytes(n_visual: Sequence[int], grid_h: int, grid_w: int, crop_h: int = 5, crop_w: int = 5) -> int:
+    return int(lib.hippo_select_workspace_bytes(len(n_visual), _host_i32(n_visual), grid_h, grid_w, crop_h, crop_w))
+
+
+def hippo_select_tokens(embeds: torch.Tensor, attn_mass: torch.Tensor, n_visual: Sequence[int], k: Sequence[int],
+                        grid_h: int, grid_w: int, crop_h: int = 5, crop_w: int = 5, score_mask: int = HIPPO_SCORE_ALL,
+                        kept_idx: Optional[torch.Tensor] = None, fused_score: Optional[torch.Tensor] = None,
+                        workspace: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """embeds [sum n_visual][d]; attn_mass fp32 [sum n_visual].  Returns (kept_idx int32 [sum k], fused fp32)."""
+    assert embeds.is_contiguous() and attn_mass.is_contiguous() and attn_mass.dtype == torch.float32
+    total = int(sum(n_visual))
+    assert embeds.shape[0] == total and attn_mass.shape[0] == total
+    if kept_idx is None:
+        kept_idx = torch.empty(max(int(sum(k)), 1), dtype=torch.int32, device=embeds.device)
+    if fused_score is None:
+        fused_score = torch.empty(total, dtype=torch.float32, device=embeds.device)
+    if workspace is None:
+        workspace = new_workspace(hippo_select_workspace_bytes(n_visual, grid_h, grid_w, crop_h, crop_w), embeds.device)
+    _check(lib.hippo_select_tokens(len(n_visual), _host_i32(n_visual), grid_h, grid_w, crop_h, crop_w, embeds.shape[1],
+                                   _dtype_code(embeds), _ptr(embeds), _ptr(attn_mass), _host_i32(k), score_mask,
+                                   _ptr(kept_idx), _ptr(fused_score), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return kept_idx[:int(sum(k))], fused_score
+
+
+# ---- gather -------------------------------------------------------------------------------------------------------
+
+def hippo_gather_kv(n_layers: int, src: KVCache, src_layer_stride_bytes: int, dst: KVCache, dst_layer_stride_bytes: int,
+                    batch: int, keep_idx: torch.Tensor, keep_offsets: torch.Tensor, total_keep: int, stream=None) -> None:
+    assert keep_idx.dtype == torch.int32 and keep_offsets.dtype == torch.int32
+    _check(lib.hippo_gather_kv(n_layers, ctypes.byref(src.struct), src_layer_stride_bytes, ctypes.byref(dst.struct),
+                               dst_layer_stride_bytes, batch, _ptr(keep_idx), _ptr(keep_offsets), int(total_keep),
+                               _stream(stream)))
+
+
+# ---- attention ----------------------------------------------------------------------------------------------------
+
+def hippo_attention_workspace_bytes(batch: int, q_len: int, n_q_heads: int, n_kv_heads: int, head_dim: int) -> int:
+    return int(lib.hippo_attention_workspace_bytes(batch, q_len, n_q_heads, n_kv_heads, head_dim))
+
+
+def _attention(fn, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse, workspace, stream):
+    assert q.is_contiguous() and q.dim() == 4 and kv_len.dtype == torch.int32
+    B, q_len, hq, d = q.shape
+    assert d == kv.head_dim and _dtype_code(q) == kv.struct.dtype
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(hippo_attention_workspace_bytes(B, q_len, hq, kv.n_kv_heads, d), q.device)
+    _check(fn(B, q_len, hq, _ptr(q), ctypes.byref(kv.struct), _ptr(kv_len), int(max_kv_len), float(softmax_scale),
+              int(num_splits), _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return out
+
+
+def hippo_verify_attention(q: torch.Tensor, kv: KVCache, kv_len: torch.Tensor, max_kv_len: int,
+                           softmax_scale: float = 0.0, num_splits: int = 0, out: Optional[torch.Tensor] = None,
+                           lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+    return _attention(lib.hippo_verify_attention, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse,
+                      workspace, stream)
+
+
+def hippo_draft_attention(q: torch.Tensor, kv: KVCache, kv_len: torch.Tensor, max_kv_len: int,
+                          softmax_scale: float = 0.0, num_splits: int = 0, out: Optional[torch.Tensor] = None,
+                          lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+    return _attention(lib.hippo_draft_attention, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse,
+                      workspace, stream)
+
+
+# ---- acceptance ---------------------------------------------------------------------------------------------------
+
+def hippo_accept_workspace_bytes(batch: int, gamma: int, vocab: int) -> int:
+    return int(lib.hippo_accept_workspace_bytes(batch, gamma, vocab))
+
+
+def hippo_accept(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                 u_accept: torch.Tensor, u_resample: torch.Tensor, n_accepted: Optional[torch.Tensor] = None,
+                 out_tokens: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None
+                 ) -> Tuple[torch.Tensor, torch.Tensor]:
+    B, g1, V = target_logits.shape
+    g = g1 - 1
+    for t in (target_logits, draft_logits, u_accept, u_resample):
+        assert t.dtype == torch.float32 and t.is_contiguous()
+    assert draft_tokens.dtype == torch.int32 and draft_tokens.is_contiguous()
+    dev = target_logits.device
+    if n_accepted is None:
+        n_accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    if out_tokens is None:
+        out_tokens = torch.empty((B, g + 1), dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = new_workspace(hippo_accept_workspace_bytes(B, g, V), dev)
+    _check(lib.hippo_accept(B, g, V, _ptr(target_logits), _ptr(draft_logits) if g else None,
+                            _ptr(draft_tokens) if g else None, _ptr(u_accept) if g else None, _ptr(u_resample), 0,
+                            _ptr(n_accepted), _ptr(out_tokens), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return n_accepted, out_tokens

@@ -1,0 +1,89 @@
+// Shared host/device helpers of the hippo CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "hippo.h"
+
+namespace hippo {
+
+constexpr int kPageSize = HIPPO_PAGE_SIZE;
+constexpr int kMaxPackedRows = HIPPO_MAX_PACKED_ROWS;
+constexpr int kNumSMs = 148;                 // B200
+constexpr size_t kWsHeaderBytes = 256;       // status word + padding
+constexpr int kExtraSlots = 4 * kNumSMs;     // partial-result slots beyond one per (sequence, kv head)
+
+// First bytes of every workspace.
+struct WsHeader {
+    int32_t status;      // 0, or HIPPO_ERR_TIMEOUT once a bounded wait gave up
+    int32_t where;       // code of the wait that gave up (debugging aid)
+    int32_t pad[62];
+};
+static_assert(sizeof(WsHeader) == kWsHeaderBytes, "header size");
+
+void set_error(const char *fmt, ...);
+int32_t fail(int32_t status, const char *fmt, ...);
+int32_t cuda_fail(cudaError_t e, const char *what);
+
+#define HIPPO_CUDA_TRY(expr)                                   \
+    do {                                                       \
+        cudaError_t e_ = (expr);                               \
+        if (e_ != cudaSuccess) return ::hippo::cuda_fail(e_, #expr); \
+    } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Layout of an attention workspace: header | arrival counters | partial slots.
+struct AttnWsLayout {
+    size_t counters_off, counters_bytes, partials_off, slot_floats, n_slots, total;
+};
+inline AttnWsLayout attn_ws_layout(int batch, int q_len, int n_q_heads, int n_kv_heads, int head_dim) {
+    AttnWsLayout L;
+    int rows = q_len * (n_q_heads / n_kv_heads);
+    L.counters_off = kWsHeaderBytes;
+    L.counters_bytes = align_up((size_t)batch * n_kv_heads * sizeof(int32_t), 256);
+    L.partials_off = L.counters_off + L.counters_bytes;
+    L.slot_floats = (size_t)rows * (head_dim + 2);
+    L.n_slots = (size_t)batch * n_kv_heads + kExtraSlots;
+    L.total = L.partials_off + align_up(L.n_slots * L.slot_floats * sizeof(float), 256);
+    return L;
+}
+
+// Arguments shared by the attention kernels.
+struct AttnParams {
+    const void *q;
+    void *out;
+    float *lse;
+    const void *k_pages;
+    const void *v_pages;
+    const int32_t *page_table;   // may be null: identity
+    const int32_t *kv_len;
+    WsHeader *header;
+    int32_t *counters;
+    float *partials;             // n_slots x (rows*(D+2)) floats: m[rows], l[rows], O[rows][D]
+    int batch, q_len, n_q_heads, n_kv_heads, head_dim, group, rows;
+    int n_pages, max_pages_per_seq, max_kv_len;
+    int num_splits;
+    float scale;
+};
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void store_from_float(float *p, float x) { *p = x; }
+__device__ __forceinline__ void store_from_float(__nv_bfloat16 *p, float x) { *p = __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ int page_of(const int32_t *page_table, int max_pages_per_seq, int b, int logical_page) {
+    return page_table ? page_table[(size_t)b * max_pages_per_seq + logical_page] : b * max_pages_per_seq + logical_page;
+}
+
+// entry points implemented per translation unit
+int32_t launch_attn_generic(const AttnParams &p, int dtype, cudaStream_t stream);
+int32_t launch_attn_combine(const AttnParams &p, int dtype, int n_splits, cudaStream_t stream);
+int32_t launch_attn_tc(const AttnParams &p, bool draft_policy, cudaStream_t stream);
+bool attn_tc_supported(const AttnParams &p, int dtype);
+
+}  // namespace hippo

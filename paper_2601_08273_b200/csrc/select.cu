@@ -1,0 +1,347 @@
+// hippo_select_tokens: semantic-aware visual-token preservation (Section 4.1).
+//
+//   Eq. 3-4  s_temp(j) = 1 - mean over the adjacent frames that contain j's grid cell of cos(v_j^f, v_j^f')
+//   Eq. 5-6  s_spa(j)  = (1/M) sum_k (S_jk - mu_j)^2 over the M tokens of j's crop, S = cosine Gram matrix, S_jj = 1
+//   Eq. 7    fused = z(attn) + z(spa) + z(temp), z = per-frame standardisation with the population sigma
+//   top-k    k best over the sequence by (fused as fp32 descending, index ascending), emitted ascending
+//
+// The standardisation of s_spa divides by a sigma of ~1e-4 on near-orthogonal embeddings, which magnifies any
+// rounding in the Gram entries by four orders of magnitude.  All dot products, crop statistics and frame
+// statistics are therefore accumulated in fp64 (bf16 x bf16 products are exact in fp64), so the kept set only
+// depends on the final rounding of the fused score to fp32.
+//
+// Kernels:  dots (norms + next-frame dot, one warp per token)  ->  spatial (one CTA per crop)  ->
+//           fuse (one CTA per frame: s_temp, three standardisations, sum)  ->  topk (one CTA per sequence,
+//           8-bit radix select on order-preserving keys, ordered compaction).
+#include <math.h>
+
+#include "common.cuh"
+
+namespace hippo {
+
+constexpr int kMaxCrop = 32;       // tokens per crop
+constexpr int kSelMaxBatch = 64;   // sequences per call (kernel-parameter tables)
+
+struct SelectParams {
+    const void *embeds;
+    const float *attn_mass;
+    float *fused;
+    int32_t *kept;
+    double *norm2, *tdot, *s_spa;   // [total tokens]
+    int batch, grid_h, grid_w, crop_h, crop_w, d, tpf, crops_y, crops_x;
+    unsigned mask;
+    int seq_off[kSelMaxBatch + 1];    // token offset of each sequence
+    int frame_off[kSelMaxBatch + 1];  // frame offset of each sequence
+    int k[kSelMaxBatch];
+    int k_off[kSelMaxBatch + 1];
+};
+
+__device__ __forceinline__ double ld_as_double(const float *p, size_t i) { return (double)p[i]; }
+__device__ __forceinline__ double ld_as_double(const __nv_bfloat16 *p, size_t i) { return (double)__bfloat162float(p[i]); }
+
+__device__ __forceinline__ double warp_sum(double v) {
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Sum over the block, result valid in every thread.  Fixed reduction order.
+__device__ double block_sum(double v, double *scratch /* [32] shared */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int w = 0; w < nw; ++w) t += scratch[w];
+    return t;
+}
+
+__device__ __forceinline__ int find_seq(const int *off, int n, int x) {  // largest b with off[b] <= x
+    int b = 0;
+    while (b + 1 < n && off[b + 1] <= x) ++b;
+    return b;
+}
+
+// ---- norms and the dot product with the same cell of the next frame ------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) select_dots_kernel(const SelectParams p) {
+    const int total = p.seq_off[p.batch];
+    const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (j >= total) return;
+    const int b = find_seq(p.seq_off, p.batch, j);
+    const T *E = (const T *)p.embeds;
+    const size_t a = (size_t)j * p.d;
+    const bool has_next = j + p.tpf < p.seq_off[b + 1];
+    const size_t c = a + (size_t)p.tpf * p.d;
+    double n2 = 0.0, td = 0.0;
+    for (int i = lane; i < p.d; i += 32) {
+        const double x = ld_as_double(E, a + i);
+        n2 = fma(x, x, n2);
+        if (has_next) td = fma(x, ld_as_double(E, c + i), td);
+    }
+    n2 = warp_sum(n2);
+    td = warp_sum(td);
+    if (lane == 0) { p.norm2[j] = n2; p.tdot[j] = td; }
+}
+
+// ---- spatial score: one CTA per crop ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) select_spatial_kernel(const SelectParams p) {
+    __shared__ int tok[kMaxCrop];
+    __shared__ double S[kMaxCrop][kMaxCrop + 1];
+    __shared__ int s_M;
+    const int crops_per_frame = p.crops_y * p.crops_x;
+    const int gframe = blockIdx.x / crops_per_frame, cr = blockIdx.x % crops_per_frame;
+    const int b = find_seq(p.frame_off, p.batch, gframe);
+    const int f = gframe - p.frame_off[b];
+    const int n_v = p.seq_off[b + 1] - p.seq_off[b];
+    const int nf = min(p.tpf, n_v - f * p.tpf);
+    const int y0 = (cr / p.crops_x) * p.crop_h, x0 = (cr % p.crops_x) * p.crop_w;
+    if (threadIdx.x == 0) {
+        int M = 0;
+        for (int y = y0; y < y0 + p.crop_h && y < p.grid_h; ++y)
+            for (int x = x0; x < x0 + p.crop_w && x < p.grid_w; ++x)
+                if (y * p.grid_w + x < nf) tok[M++] = p.seq_off[b] + f * p.tpf + y * p.grid_w + x;
+        s_M = M;
+    }
+    __syncthreads();
+    const int M = s_M;
+    if (M == 0) return;
+    const T *E = (const T *)p.embeds;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    // upper triangle (a < b) of the raw Gram matrix in fp64; norms come from the dots kernel
+    const int n_pairs = M * (M - 1) / 2;
+    for (int pr = warp; pr < n_pairs; pr += nw) {
+        int a = 0, rem = pr;
+        while (rem >= M - 1 - a) { rem -= M - 1 - a; ++a; }
+        const int c = a + 1 + rem;
+        const size_t oa = (size_t)tok[a] * p.d, oc = (size_t)tok[c] * p.d;
+        double acc = 0.0;
+        for (int i = lane; i < p.d; i += 32) acc = fma(ld_as_double(E, oa + i), ld_as_double(E, oc + i), acc);
+        acc = warp_sum(acc);
+        if (lane == 0) {
+            const double na = p.norm2[tok[a]], nc = p.norm2[tok[c]];
+            const double s = (na > 0.0 && nc > 0.0) ? acc / (sqrt(na) * sqrt(nc)) : 0.0;
+            S[a][c] = s;
+            S[c][a] = s;
+        }
+    }
+    if (threadIdx.x < M) S[threadIdx.x][threadIdx.x] = 1.0;
+    __syncthreads();
+    if (threadIdx.x < M) {
+        const int a = threadIdx.x;
+        double mu = 0.0;
+        for (int c = 0; c < M; ++c) mu += S[a][c];
+        mu /= M;
+        double var = 0.0;
+        for (int c = 0; c < M; ++c) var += (S[a][c] - mu) * (S[a][c] - mu);
+        p.s_spa[tok[a]] = var / M;
+    }
+}
+
+// ---- per-frame standardisation and fusion: one CTA per frame ---------------------------------------------------
+__device__ double standardise(double x, bool valid, int n, double *scratch) {
+    const double mu = block_sum(valid ? x : 0.0, scratch) / n;
+    const double dv = valid ? x - mu : 0.0;
+    const double var = block_sum(dv * dv, scratch) / n;
+    const double floor_ = 1e-24 * fmax(1.0, mu * mu);
+    if (var <= floor_) return 0.0;
+    return dv / sqrt(var);
+}
+
+__global__ void __launch_bounds__(1024) select_fuse_kernel(const SelectParams p) {
+    __shared__ double scratch[32];
+    const int gframe = blockIdx.x;
+    const int b = find_seq(p.frame_off, p.batch, gframe);
+    const int f = gframe - p.frame_off[b];
+    const int n_v = p.seq_off[b + 1] - p.seq_off[b];
+    const int n_frames = (n_v + p.tpf - 1) / p.tpf;
+    const int nf = min(p.tpf, n_v - f * p.tpf);
+    // blockDim.x >= tokens per frame (checked on the host): thread c owns grid cell c
+    const int c = threadIdx.x;
+    const bool valid = c < nf;
+    const int j = p.seq_off[b] + f * p.tpf + c;
+    double fused = 0.0;
+    if (p.mask & HIPPO_SCORE_ATTN) fused += standardise(valid ? (double)p.attn_mass[j] : 0.0, valid, nf, scratch);
+    if (p.mask & HIPPO_SCORE_SPA) fused += standardise(valid ? p.s_spa[j] : 0.0, valid, nf, scratch);
+    if (p.mask & HIPPO_SCORE_TEMP) {
+        double st = 0.0;
+        if (valid) {
+            double sum = 0.0;
+            int cnt = 0;
+            const double nj = p.norm2[j];
+            if (f > 0) {  // previous frame always holds every cell
+                const double nk = p.norm2[j - p.tpf];
+                sum += (nj > 0.0 && nk > 0.0) ? p.tdot[j - p.tpf] / (sqrt(nj) * sqrt(nk)) : 0.0;
+                ++cnt;
+            }
+            if (f + 1 < n_frames && c < min(p.tpf, n_v - (f + 1) * p.tpf)) {
+                const double nk = p.norm2[j + p.tpf];
+                sum += (nj > 0.0 && nk > 0.0) ? p.tdot[j] / (sqrt(nj) * sqrt(nk)) : 0.0;
+                ++cnt;
+            }
+            st = 1.0 - (cnt ? sum / cnt : 0.0);
+        }
+        fused += standardise(st, valid, nf, scratch);
+    }
+    if (valid) p.fused[j] = (float)fused;
+}
+
+// ---- top-k: one CTA per sequence --------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t order_key(float x) {  // larger float -> larger key
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p) {
+    __shared__ int hist[256];
+    __shared__ int warp_cnt[32];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_remaining, s_base_eq, s_base_out;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = p.seq_off[b + 1] - p.seq_off[b];
+    const int k = p.k[b];
+    if (k <= 0) return;
+    const float *score = p.fused + p.seq_off[b];
+    int32_t *out = p.kept + p.k_off[b];
+    // radix select: find the key T of the k-th largest element
+    if (tid == 0) { s_prefix = 0; s_remaining = k; }
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        for (int i = tid; i < 256; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+        for (int i = tid; i < n; i += blockDim.x) {
+            const uint32_t key = order_key(score[i]);
+            if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int rem = s_remaining, bin = 255;
+            for (; bin > 0; --bin) {
+                if (hist[bin] >= rem) break;
+                rem -= hist[bin];
+            }
+            s_prefix = prefix | ((uint32_t)bin << shift);
+            s_remaining = rem;  // how many of the elements inside this bin are still needed
+        }
+        __syncthreads();
+    }
+    const uint32_t T = s_prefix;
+    const int need_eq = s_remaining;  // elements equal to T to keep: those with the smallest indices
+    if (tid == 0) { s_base_eq = 0; s_base_out = 0; }
+    __syncthreads();
+    // ordered compaction, blockDim.x elements at a time
+    for (int start = 0; start < n; start += blockDim.x) {
+        const int i = start + tid;
+        const uint32_t key = i < n ? order_key(score[i]) : 0u;
+        const bool gt = i < n && key > T, eq = i < n && key == T;
+        // rank of this element among the equal ones (exclusive, in index order)
+        unsigned bal = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) warp_cnt[warp] = __popc(bal);
+        __syncthreads();
+        int eq_rank = s_base_eq + __popc(bal & ((1u << lane) - 1));
+        int eq_total = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { if (w < warp) eq_rank += warp_cnt[w]; eq_total += warp_cnt[w]; }
+        const bool sel = gt || (eq && eq_rank < need_eq);
+        __syncthreads();
+        bal = __ballot_sync(0xffffffffu, sel);
+        if (lane == 0) warp_cnt[warp] = __popc(bal);
+        __syncthreads();
+        int pos = s_base_out + __popc(bal & ((1u << lane) - 1));
+        int sel_total = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { if (w < warp) pos += warp_cnt[w]; sel_total += warp_cnt[w]; }
+        if (sel && pos < k) out[pos] = i;
+        __syncthreads();
+        if (tid == 0) { s_base_eq += eq_total; s_base_out += sel_total; }
+        __syncthreads();
+    }
+}
+
+struct SelectWs { size_t norm2_off, tdot_off, spa_off, total; };
+static SelectWs select_ws(long long total_tokens) {
+    SelectWs w;
+    const size_t a = align_up((size_t)total_tokens * sizeof(double), 256);
+    w.norm2_off = kWsHeaderBytes;
+    w.tdot_off = w.norm2_off + a;
+    w.spa_off = w.tdot_off + a;
+    w.total = w.spa_off + a;
+    return w;
+}
+
+}  // namespace hippo
+
+extern "C" {
+
+size_t hippo_select_workspace_bytes(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w,
+                                    int32_t crop_h, int32_t crop_w) {
+    (void)grid_h; (void)grid_w; (void)crop_h; (void)crop_w;
+    if (batch <= 0 || !n_visual) return 0;
+    long long t = 0;
+    for (int b = 0; b < batch; ++b) { if (n_visual[b] <= 0) return 0; t += n_visual[b]; }
+    return hippo::select_ws(t).total;
+}
+
+int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w, int32_t crop_h,
+                            int32_t crop_w, int32_t embed_dim, int32_t dtype, const void *embeds,
+                            const float *attn_mass, const int32_t *k, uint32_t score_mask, int32_t *kept_idx,
+                            float *fused_score, void *workspace, size_t workspace_bytes, void *stream) {
+    using namespace hippo;
+    const char *who = "hippo_select_tokens";
+    if (batch <= 0 || !n_visual || !k) return fail(HIPPO_ERR_INVALID_ARG, "%s: bad batch / null host arrays", who);
+    if (batch > kSelMaxBatch) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: batch > %d", who, kSelMaxBatch);
+    if (grid_h <= 0 || grid_w <= 0 || crop_h <= 0 || crop_w <= 0 || embed_dim <= 0)
+        return fail(HIPPO_ERR_INVALID_ARG, "%s: non-positive geometry", who);
+    if (dtype != HIPPO_DTYPE_FP32 && dtype != HIPPO_DTYPE_BF16) return fail(HIPPO_ERR_INVALID_ARG, "%s: unknown dtype", who);
+    if (crop_h * crop_w > kMaxCrop) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: crop larger than %d tokens", who, kMaxCrop);
+    if ((long long)grid_h * grid_w > 1024) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: more than 1024 tokens per frame", who);
+    if (embed_dim % 8) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: embed_dim must be a multiple of 8", who);
+    if (!embeds || !attn_mass || !fused_score || !workspace) return fail(HIPPO_ERR_INVALID_ARG, "%s: null pointer", who);
+    if ((score_mask & ~HIPPO_SCORE_ALL) != 0) return fail(HIPPO_ERR_INVALID_ARG, "%s: unknown score_mask bits", who);
+    if ((uintptr_t)workspace & 255) return fail(HIPPO_ERR_INVALID_ARG, "%s: workspace must be 256-byte aligned", who);
+    if ((uintptr_t)embeds & 15) return fail(HIPPO_ERR_INVALID_ARG, "%s: embeds must be 16-byte aligned", who);
+
+    SelectParams p;
+    p.tpf = grid_h * grid_w;
+    long long tok = 0, frames = 0, ksum = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (n_visual[b] <= 0) return fail(HIPPO_ERR_INVALID_ARG, "%s: n_visual[%d] <= 0", who, b);
+        if (k[b] < 0 || k[b] > n_visual[b]) return fail(HIPPO_ERR_INVALID_ARG, "%s: k[%d] outside [0, n_visual]", who, b);
+        p.seq_off[b] = (int)tok; p.frame_off[b] = (int)frames; p.k[b] = k[b]; p.k_off[b] = (int)ksum;
+        tok += n_visual[b]; frames += (n_visual[b] + p.tpf - 1) / p.tpf; ksum += k[b];
+        if (tok > 0x7fffffffLL / 2) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: too many tokens", who);
+    }
+    p.seq_off[batch] = (int)tok; p.frame_off[batch] = (int)frames; p.k_off[batch] = (int)ksum;
+    if (ksum > 0 && !kept_idx) return fail(HIPPO_ERR_INVALID_ARG, "%s: null kept_idx", who);
+    SelectWs w = select_ws(tok);
+    if (workspace_bytes < w.total) return fail(HIPPO_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu bytes", who, workspace_bytes, w.total);
+    p.embeds = embeds; p.attn_mass = attn_mass; p.fused = fused_score; p.kept = kept_idx;
+    p.norm2 = (double *)((char *)workspace + w.norm2_off);
+    p.tdot = (double *)((char *)workspace + w.tdot_off);
+    p.s_spa = (double *)((char *)workspace + w.spa_off);
+    p.batch = batch; p.grid_h = grid_h; p.grid_w = grid_w; p.crop_h = crop_h; p.crop_w = crop_w; p.d = embed_dim;
+    p.crops_y = ceil_div(grid_h, crop_h); p.crops_x = ceil_div(grid_w, crop_w);
+    p.mask = score_mask;
+    cudaStream_t s = (cudaStream_t)stream;
+    const bool need_emb = (score_mask & (HIPPO_SCORE_TEMP | HIPPO_SCORE_SPA)) != 0;
+    if (need_emb) {
+        const int warps = 8;
+        dim3 g1((unsigned)((tok + warps - 1) / warps));
+        if (dtype == HIPPO_DTYPE_FP32) select_dots_kernel<float><<<g1, warps * 32, 0, s>>>(p);
+        else select_dots_kernel<__nv_bfloat16><<<g1, warps * 32, 0, s>>>(p);
+    }
+    if (score_mask & HIPPO_SCORE_SPA) {
+        dim3 g2((unsigned)(frames * p.crops_y * p.crops_x));
+        if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float><<<g2, 256, 0, s>>>(p);
+        else select_spatial_kernel<__nv_bfloat16><<<g2, 256, 0, s>>>(p);
+    }
+    const int fuse_threads = ((p.tpf + 31) / 32) * 32;
+    select_fuse_kernel<<<(unsigned)frames, fuse_threads, 0, s>>>(p);
+    if (ksum > 0) select_topk_kernel<<<batch, 1024, 0, s>>>(p);
+    HIPPO_CUDA_TRY(cudaGetLastError());
+    return HIPPO_OK;
+}
+
+}  // extern "C"

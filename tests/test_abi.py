@@ -1,0 +1,55 @@
+"""The C-ABI library builds, loads without a GPU and exports every symbol include/hippo.h declares; argument
+validation rejects bad calls before anything is launched.  CPU only."""
+import ctypes
+import os
+import re
+
+from paper_2601_08273_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "hippo.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hippo_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    build.build_library()
+    from paper_2601_08273_b200 import binding
+    names = declared_functions()
+    assert {"hippo_select_tokens", "hippo_gather_kv", "hippo_draft_attention", "hippo_verify_attention",
+            "hippo_accept"} <= set(names)
+    for n in names:
+        assert hasattr(binding.lib, n), n
+    assert binding.hippo_version() == 100
+    assert binding.lib.hippo_status_string(-5).decode() == "device-side wait timed out"
+
+
+def test_argument_validation_happens_before_any_launch():
+    from paper_2601_08273_b200 import binding as hb
+    lib = hb.lib
+    assert lib.hippo_accept(0, 1, 10, None, None, None, None, None, 0, None, None, None, 0, None) == hb.HIPPO_ERR_INVALID_ARG
+    assert lib.hippo_accept(1, 1, 10, None, None, None, None, None, 0, None, None, None, 0, None) == hb.HIPPO_ERR_INVALID_ARG
+    assert b"null pointer" in lib.hippo_last_error()
+    assert lib.hippo_accept(1, 1, 10, 256, 256, 256, 256, 256, 7, 256, 256, 256, 1 << 20, None) == hb.HIPPO_ERR_UNIMPLEMENTED
+    assert lib.hippo_accept(1, 1, 10, 256, 256, 256, 256, 256, 0, 256, 256, 256, 16, None) == hb.HIPPO_ERR_WORKSPACE_TOO_SMALL
+    kv = hb.KVCacheStruct(ctypes.sizeof(hb.KVCacheStruct), hb.HIPPO_DTYPE_BF16, 2, 64, 10, 4, 1024, 2048, None)
+    args = lambda **o: [o.get("B", 1), o.get("q_len", 1), o.get("hq", 14), 256, ctypes.byref(kv), 256,
+                        o.get("max_kv", 200), 0.0, 0, 256, None, o.get("ws", 256), o.get("ws_bytes", 1 << 30), None]
+    assert lib.hippo_draft_attention(*args(hq=15)) == hb.HIPPO_ERR_INVALID_ARG          # 15 % 2 != 0
+    assert lib.hippo_draft_attention(*args(max_kv=257)) == hb.HIPPO_ERR_INVALID_ARG      # > 4 pages
+    assert lib.hippo_draft_attention(*args(ws_bytes=1000)) == hb.HIPPO_ERR_WORKSPACE_TOO_SMALL
+    assert lib.hippo_draft_attention(*args(q_len=40)) == hb.HIPPO_ERR_UNSUPPORTED_SHAPE  # 40*7 packed rows
+    assert lib.hippo_draft_attention(*args(B=3)) == hb.HIPPO_ERR_INVALID_ARG             # identity mapping needs 12 pages
+    kv.struct_size = 8
+    assert lib.hippo_verify_attention(*args()) == hb.HIPPO_ERR_INVALID_ARG
+    n_visual = (ctypes.c_int32 * 1)(100)
+    k = (ctypes.c_int32 * 1)(101)
+    assert lib.hippo_select_tokens(1, n_visual, 14, 14, 5, 5, 64, 1, 256, 256, k, 7, 256, 256, 256, 1 << 30, None) == hb.HIPPO_ERR_INVALID_ARG
+    k[0] = 10
+    assert lib.hippo_select_tokens(1, n_visual, 14, 14, 6, 6, 64, 1, 256, 256, k, 7, 256, 256, 256, 1 << 30, None) == hb.HIPPO_ERR_UNSUPPORTED_SHAPE
+    assert hb.hippo_select_workspace_bytes([100], 14, 14) >= 256 + 3 * 800
+    assert hb.hippo_attention_workspace_bytes(1, 6, 28, 4, 128) > 42 * 130 * 4 * 4
+    assert hb.hippo_accept_workspace_bytes(1, 5, 152064) > 0

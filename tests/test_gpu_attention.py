@@ -1,0 +1,161 @@
+"""GPU parity: hippo_verify_attention / hippo_draft_attention (through the C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import TOL, assert_close, dev, host, paged_cache
+from paper_2601_08273_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def hb():
+    from paper_2601_08273_b200 import binding
+    return binding
+
+
+def run_case(hb, fn, q, k, v, lens, dtype, shuffle_seed=None, num_splits=0, want_lse=True, fill=0.0, spare=0):
+    kv, _, _ = paged_cache(hb, k, v, lens, dtype, shuffle_seed=shuffle_seed, fill=fill, spare=spare)
+    qd = dev(q, dtype)
+    kvl = dev(np.asarray(lens, np.int32))
+    lse = torch.full(q.shape[:3], float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
+    out = fn(qd, kv, kvl, max(lens), num_splits=num_splits, lse=lse)
+    torch.cuda.synchronize()
+    return host(out), (None if lse is None else host(lse))
+
+
+def check_full(hb, fn, q, k, v, lens, dtype, **kw):
+    got, lse = run_case(hb, fn, q, k, v, lens, dtype, **kw)
+    ref, ref_lse = oracle.attention(q, k, v, lens)
+    assert_close(got, ref, TOL[dtype], "attention out")
+    if lse is not None:
+        assert_close(lse, ref_lse, TOL[dtype] if dtype == "fp32" else 2e-3, "lse")
+    return got
+
+
+def test_c0_verify_and_draft_fp32(hb):
+    cfg = W.CONFIGS[0]
+    n_v = W.visual_lengths(cfg)[0]
+    q_len = cfg.gamma + 1
+    lens = [n_v + cfg.n_text + q_len]
+    inp = W.attention_inputs(cfg, "target", lens, q_len)
+    check_full(hb, hb.hippo_verify_attention, inp["q"], inp["k"], inp["v"], lens, "fp32")
+    # draft: pruned context (26 kept + 32 text) plus the tokens drafted so far, one query token
+    for step in range(cfg.gamma):
+        lens_d = [W.keep_count(n_v, cfg.keep_pct) + cfg.n_text + step + 1]
+        inp = W.attention_inputs(cfg, "draft", lens_d, 1, layer=step)
+        check_full(hb, hb.hippo_draft_attention, inp["q"], inp["k"], inp["v"], lens_d, "fp32")
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("D", [64, 128])
+def test_ragged_batch_paged_several_tiles(hb, dtype, D):
+    rng = np.random.default_rng(17)
+    B, q_len, Hq, Hkv = 3, 6, 8, 2
+    lens = [333, 6, 129]          # several tiles + ragged tail, kv_len == q_len, one key past a page boundary
+    q = W.round_to_storage(rng.standard_normal((B, q_len, Hq, D)).astype(np.float32), dtype)
+    k = W.round_to_storage(rng.standard_normal((B, max(lens), Hkv, D)).astype(np.float32), dtype)
+    v = W.round_to_storage(rng.standard_normal((B, max(lens), Hkv, D)).astype(np.float32), dtype)
+    a = check_full(hb, hb.hippo_verify_attention, q, k, v, lens, dtype, shuffle_seed=5, spare=3)
+    # slots past each length hold NaN: they must never be read into a result
+    b = check_full(hb, hb.hippo_verify_attention, q, k, v, lens, dtype, shuffle_seed=5, spare=3, fill=np.nan)
+    np.testing.assert_array_equal(a, b)
+    # different physical page order, same result bit for bit
+    c = check_full(hb, hb.hippo_verify_attention, q, k, v, lens, dtype, shuffle_seed=6)
+    np.testing.assert_array_equal(a, c)
+    # split count does not matter beyond rounding
+    for s in (1, 2, 5):
+        check_full(hb, hb.hippo_verify_attention, q, k, v, lens, dtype, shuffle_seed=5, num_splits=s)
+    check_full(hb, hb.hippo_draft_attention, q[:, :1], k, v, lens, dtype, shuffle_seed=5)
+
+
+@pytest.mark.parametrize("rows", [(1, 7), (9, 8), (6, 7), (8, 4), (16, 8)])
+def test_packed_row_shapes_bf16(hb, rows):
+    q_len, G = rows
+    rng = np.random.default_rng(q_len * 100 + G)
+    Hkv, D, lens = 2, 128, [1000]
+    q = W.round_to_storage(rng.standard_normal((1, q_len, Hkv * G, D)).astype(np.float32), "bf16")
+    k = W.round_to_storage(rng.standard_normal((1, lens[0], Hkv, D)).astype(np.float32), "bf16")
+    v = W.round_to_storage(rng.standard_normal((1, lens[0], Hkv, D)).astype(np.float32), "bf16")
+    check_full(hb, hb.hippo_verify_attention, q, k, v, lens, "bf16")
+
+
+def test_short_sequence_is_skipped_and_zeroed(hb):
+    rng = np.random.default_rng(3)
+    B, q_len, Hq, Hkv, D = 2, 4, 4, 2, 64
+    lens = [2, 70]               # first sequence shorter than q_len
+    q = rng.standard_normal((B, q_len, Hq, D)).astype(np.float32)
+    k = rng.standard_normal((B, 70, Hkv, D)).astype(np.float32)
+    v = rng.standard_normal((B, 70, Hkv, D)).astype(np.float32)
+    got, lse = run_case(hb, hb.hippo_verify_attention, q, k, v, lens, "fp32", shuffle_seed=1)
+    assert np.all(got[0] == 0) and np.all(np.isneginf(lse[0]))
+    ref, _ = oracle.attention(q[1:], k[1:], v[1:], lens[1:])
+    assert_close(got[1:], ref, 1e-5)
+
+
+def sampled_rows(rng, B, q_len, Hq, n):
+    rows = {(0, 0, 0), (B - 1, q_len - 1, Hq - 1)}
+    while len(rows) < n:
+        rows.add((int(rng.integers(B)), int(rng.integers(q_len)), int(rng.integers(Hq))))
+    return sorted(rows)
+
+
+@pytest.mark.parametrize("ci", [1, 2, 4])
+def test_full_size_verify_sampled_rows(hb, ci):
+    cfg = W.CONFIGS[ci]
+    n_v = W.visual_lengths(cfg)[0]
+    gammas = W.C4_GAMMA_SWEEP if ci == 4 else (cfg.gamma,)
+    for g in gammas:
+        q_len = g + 1
+        lens = [n_v + cfg.n_text + q_len]
+        inp = W.attention_inputs(cfg, "target", lens, q_len)
+        got, lse = run_case(hb, hb.hippo_verify_attention, inp["q"], inp["k"], inp["v"], lens, cfg.dtype)
+        rows = sampled_rows(np.random.default_rng(ci), 1, q_len, cfg.tgt_q_heads, 24)
+        ref, ref_lse = oracle.attention(inp["q"], inp["k"], inp["v"], lens, rows=rows)
+        sel = np.array(rows)
+        assert_close(got[sel[:, 0], sel[:, 1], sel[:, 2]], ref, TOL[cfg.dtype], "c%d gamma %d" % (ci, g))
+        assert_close(lse[sel[:, 0], sel[:, 1], sel[:, 2]], ref_lse, 2e-3, "lse")
+        assert np.isfinite(got).all()
+
+
+def test_c3_batched_paged_verify_and_draft(hb):
+    cfg = W.CONFIGS[3]
+    q_len = cfg.gamma + 1
+    n_vs = W.visual_lengths(cfg)
+    lens = [n + cfg.n_text + q_len for n in n_vs]
+    inp = W.attention_inputs(cfg, "target", lens, q_len)
+    got, _ = run_case(hb, hb.hippo_verify_attention, inp["q"], inp["k"], inp["v"], lens, cfg.dtype, shuffle_seed=33)
+    rows = sampled_rows(np.random.default_rng(3), cfg.batch, q_len, cfg.tgt_q_heads, 32)
+    ref, _ = oracle.attention(inp["q"], inp["k"], inp["v"], lens, rows=rows)
+    sel = np.array(rows)
+    assert_close(got[sel[:, 0], sel[:, 1], sel[:, 2]], ref, TOL[cfg.dtype], "c3 verify")
+    lens_d = [W.keep_count(n, cfg.keep_pct) + cfg.n_text + 1 for n in n_vs]
+    inp = W.attention_inputs(cfg, "draft", lens_d, 1)
+    got, _ = run_case(hb, hb.hippo_draft_attention, inp["q"], inp["k"], inp["v"], lens_d, cfg.dtype, shuffle_seed=34)
+    ref, _ = oracle.attention(inp["q"], inp["k"], inp["v"], lens_d)
+    assert_close(got, ref, TOL[cfg.dtype], "c3 draft")
+
+
+@pytest.mark.parametrize("ci", [1, 2, 4])
+def test_full_size_draft(hb, ci):
+    cfg = W.CONFIGS[ci]
+    n_v = W.visual_lengths(cfg)[0]
+    pcts = W.C4_KEEP_PCT_SWEEP if ci == 4 else (cfg.keep_pct,)
+    for pct in pcts:
+        lens = [W.keep_count(n_v, pct) + cfg.n_text + cfg.gamma]
+        inp = W.attention_inputs(cfg, "draft", lens, 1)
+        got, _ = run_case(hb, hb.hippo_draft_attention, inp["q"], inp["k"], inp["v"], lens, cfg.dtype)
+        ref, _ = oracle.attention(inp["q"], inp["k"], inp["v"], lens)
+        assert_close(got, ref, TOL[cfg.dtype], "c%d draft keep %d%%" % (ci, pct))
+
+
+def test_workspace_status_is_clean(hb):
+    ws = hb.new_workspace(hb.hippo_attention_workspace_bytes(1, 2, 4, 2, 64))
+    rng = np.random.default_rng(0)
+    q = dev(rng.standard_normal((1, 2, 4, 64)).astype(np.float32), "bf16")
+    k = rng.standard_normal((1, 100, 2, 64)).astype(np.float32)
+    kv, _, _ = paged_cache(hb, k, k, [100], "bf16")
+    hb.hippo_verify_attention(q, kv, dev(np.asarray([100], np.int32)), 100, workspace=ws)
+    assert hb.hippo_workspace_status(ws) == hb.HIPPO_OK

@@ -83,6 +83,8 @@ int32_t hippo_version(void);
 const char *hippo_status_string(int32_t status);
 /* Text of the last error raised on the calling host thread (empty string if none). */
 const char *hippo_last_error(void);
+/* Kernels launched by this library in this process so far (host-side counter, all threads). */
+uint64_t hippo_launch_count(void);
 /* Synchronises `stream`, then reads the status word that kernels keep in the first bytes of `workspace`:
  * HIPPO_OK, or HIPPO_ERR_TIMEOUT if a bounded device-side wait gave up since hippo_workspace_reset(). */
 int32_t hippo_workspace_status(const void *workspace, void *stream);
@@ -104,7 +106,9 @@ int32_t hippo_workspace_reset(void *workspace, size_t workspace_bytes, void *str
  * sequence b starts at token offset sum(n_visual[0..b)).
  *   n_visual  host int32 [batch], each >= 1          k         host int32 [batch], 0 <= k[b] <= n_visual[b]
  *   embeds    [sum n_visual][embed_dim] dtype         attn_mass fp32 [sum n_visual]
- *   kept_idx  out int32 [sum k]: sequence b's indices (relative to its own start, ascending) at offset sum(k[0..b))
+ *   kept_idx  out int32: sequence b's k[b] indices (relative to its own start, ascending) are written at element
+ *             offset kept_offsets[b]; kept_offsets (host int32 [batch]) may be NULL, meaning sum(k[0..b)).  Explicit
+ *             offsets let the caller interleave other entries (e.g. always-kept text positions) in the same list.
  *   fused_score out fp32 [sum n_visual]
  * Scores are accumulated in fp64.  embed_dim must be a multiple of 8; crop_h*crop_w <= 32.
  */
@@ -112,8 +116,9 @@ size_t hippo_select_workspace_bytes(int32_t batch, const int32_t *n_visual, int3
                                     int32_t crop_h, int32_t crop_w);
 int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w, int32_t crop_h,
                             int32_t crop_w, int32_t embed_dim, int32_t dtype, const void *embeds,
-                            const float *attn_mass, const int32_t *k, uint32_t score_mask, int32_t *kept_idx,
-                            float *fused_score, void *workspace, size_t workspace_bytes, void *stream);
+                            const float *attn_mass, const int32_t *k, const int32_t *kept_offsets,
+                            uint32_t score_mask, int32_t *kept_idx, float *fused_score, void *workspace,
+                            size_t workspace_bytes, void *stream);
 
 /* ---- gather: pruning the draft KV cache (Limitations (i); experimental set-up: "remove the corresponding
  *      video features") --------------------------------------------------------------------------------------- */

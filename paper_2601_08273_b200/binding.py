@@ -50,6 +50,7 @@ lib.hippo_version.restype = _i32
 lib.hippo_status_string.restype = ctypes.c_char_p
 lib.hippo_status_string.argtypes = [_i32]
 lib.hippo_last_error.restype = ctypes.c_char_p
+lib.hippo_launch_count.restype = ctypes.c_uint64
 lib.hippo_workspace_status.restype = _i32
 lib.hippo_workspace_status.argtypes = [_vp, _vp]
 lib.hippo_workspace_reset.restype = _i32
@@ -57,7 +58,7 @@ lib.hippo_workspace_reset.argtypes = [_vp, _sz, _vp]
 lib.hippo_select_workspace_bytes.restype = _sz
 lib.hippo_select_workspace_bytes.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32]
 lib.hippo_select_tokens.restype = _i32
-lib.hippo_select_tokens.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _I32P, _u32, _vp, _vp,
+lib.hippo_select_tokens.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _I32P, _I32P, _u32, _vp, _vp,
                                     _vp, _sz, _vp]
 lib.hippo_gather_kv.restype = _i32
 lib.hippo_gather_kv.argtypes = [_i32, _KVP, _sz, _KVP, _sz, _i32, _vp, _vp, _i32, _vp]
@@ -110,6 +111,10 @@ def hippo_version() -> int:
     return int(lib.hippo_version())
 
 
+def hippo_launch_count() -> int:
+    return int(lib.hippo_launch_count())
+
+
 class KVCache:
     """Descriptor of one layer's paged cache; keeps the tensors alive.  k_pages, v_pages:
     [n_pages][n_kv_heads][64][head_dim]; page_table int32 [batch][max_pages_per_seq] or None (identity)."""
@@ -160,7 +165,8 @@ def hippo_select_workspace_bytes(n_visual: Sequence[int], grid_h: int, grid_w: i
 
 def hippo_select_tokens(embeds: torch.Tensor, attn_mass: torch.Tensor, n_visual: Sequence[int], k: Sequence[int],
                         grid_h: int, grid_w: int, crop_h: int = 5, crop_w: int = 5, score_mask: int = HIPPO_SCORE_ALL,
-                        kept_idx: Optional[torch.Tensor] = None, fused_score: Optional[torch.Tensor] = None,
+                        kept_idx: Optional[torch.Tensor] = None, kept_offsets: Optional[Sequence[int]] = None,
+                        fused_score: Optional[torch.Tensor] = None,
                         workspace: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
     """embeds [sum n_visual][d]; attn_mass fp32 [sum n_visual].  Returns (kept_idx int32 [sum k], fused fp32)."""
     assert embeds.is_contiguous() and attn_mass.is_contiguous() and attn_mass.dtype == torch.float32
@@ -173,9 +179,10 @@ def hippo_select_tokens(embeds: torch.Tensor, attn_mass: torch.Tensor, n_visual:
     if workspace is None:
         workspace = new_workspace(hippo_select_workspace_bytes(n_visual, grid_h, grid_w, crop_h, crop_w), embeds.device)
     _check(lib.hippo_select_tokens(len(n_visual), _host_i32(n_visual), grid_h, grid_w, crop_h, crop_w, embeds.shape[1],
-                                   _dtype_code(embeds), _ptr(embeds), _ptr(attn_mass), _host_i32(k), score_mask,
+                                   _dtype_code(embeds), _ptr(embeds), _ptr(attn_mass), _host_i32(k),
+                                   None if kept_offsets is None else _host_i32(kept_offsets), score_mask,
                                    _ptr(kept_idx), _ptr(fused_score), _ptr(workspace), workspace.numel(), _stream(stream)))
-    return kept_idx[:int(sum(k))], fused_score
+    return (kept_idx[:int(sum(k))] if kept_offsets is None else kept_idx), fused_score
 
 
 # ---- gather -------------------------------------------------------------------------------------------------------

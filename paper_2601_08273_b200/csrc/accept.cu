@@ -285,6 +285,7 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
     accept_decide_kernel<<<batch, kAccThreads, (2 * gamma + 1) * 2 * sizeof(double), s>>>(p);
     accept_wsum_kernel<<<dim3(w.n_chunks, batch), kAccThreads, 0, s>>>(p);
     accept_pick_kernel<<<batch, kAccThreads, 0, s>>>(p);
+    count_launches(4);
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;
 }

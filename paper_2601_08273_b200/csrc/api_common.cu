@@ -2,11 +2,17 @@
 #include <stdarg.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace hippo {
 
 static thread_local char g_err[512] = {0};
+static std::atomic<unsigned long long> g_launches{0};
+
+void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+unsigned long long launches() { return g_launches.load(std::memory_order_relaxed); }
 
 void set_error(const char *fmt, ...) {
     va_list ap;
@@ -48,6 +54,8 @@ const char *hippo_status_string(int32_t status) {
 }
 
 const char *hippo_last_error(void) { return hippo::g_err; }
+
+uint64_t hippo_launch_count(void) { return (uint64_t)hippo::launches(); }
 
 int32_t hippo_workspace_status(const void *workspace, void *stream) {
     if (!workspace) return hippo::fail(HIPPO_ERR_INVALID_ARG, "hippo_workspace_status: null workspace");

@@ -148,6 +148,7 @@ int32_t launch_attn_generic(const AttnParams &p, int dtype, cudaStream_t stream)
         HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_generic_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attn_generic_kernel<__nv_bfloat16><<<grid, kGenThreads, smem, stream>>>(p);
     }
+    count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     return launch_attn_combine(p, dtype, p.num_splits, stream);
 }
@@ -160,6 +161,7 @@ int32_t launch_attn_combine(const AttnParams &p, int dtype, int n_splits, cudaSt
         attn_combine_kernel<float><<<grid, warps_per_block * 32, 0, stream>>>(p, n_splits);
     else
         attn_combine_kernel<__nv_bfloat16><<<grid, warps_per_block * 32, 0, stream>>>(p, n_splits);
+    count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;
 }

@@ -24,6 +24,8 @@ struct WsHeader {
 };
 static_assert(sizeof(WsHeader) == kWsHeaderBytes, "header size");
 
+// Number of kernels this library has launched in this process (diagnostics; see hippo_launch_count()).
+void count_launches(int n);
 void set_error(const char *fmt, ...);
 int32_t fail(int32_t status, const char *fmt, ...);
 int32_t cuda_fail(cudaError_t e, const char *what);

@@ -97,6 +97,7 @@ extern "C" int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src
     const long long cap = (long long)kNumSMs * 32;
     if (blocks > cap) blocks = cap;
     gather_kv_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(p);
+    count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;
 }

@@ -286,8 +286,9 @@ size_t hippo_select_workspace_bytes(int32_t batch, const int32_t *n_visual, int3
 
 int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w, int32_t crop_h,
                             int32_t crop_w, int32_t embed_dim, int32_t dtype, const void *embeds,
-                            const float *attn_mass, const int32_t *k, uint32_t score_mask, int32_t *kept_idx,
-                            float *fused_score, void *workspace, size_t workspace_bytes, void *stream) {
+                            const float *attn_mass, const int32_t *k, const int32_t *kept_offsets,
+                            uint32_t score_mask, int32_t *kept_idx, float *fused_score, void *workspace,
+                            size_t workspace_bytes, void *stream) {
     using namespace hippo;
     const char *who = "hippo_select_tokens";
     if (batch <= 0 || !n_visual || !k) return fail(HIPPO_ERR_INVALID_ARG, "%s: bad batch / null host arrays", who);
@@ -309,7 +310,9 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
     for (int b = 0; b < batch; ++b) {
         if (n_visual[b] <= 0) return fail(HIPPO_ERR_INVALID_ARG, "%s: n_visual[%d] <= 0", who, b);
         if (k[b] < 0 || k[b] > n_visual[b]) return fail(HIPPO_ERR_INVALID_ARG, "%s: k[%d] outside [0, n_visual]", who, b);
-        p.seq_off[b] = (int)tok; p.frame_off[b] = (int)frames; p.k[b] = k[b]; p.k_off[b] = (int)ksum;
+        p.seq_off[b] = (int)tok; p.frame_off[b] = (int)frames; p.k[b] = k[b];
+        if (kept_offsets && kept_offsets[b] < 0) return fail(HIPPO_ERR_INVALID_ARG, "%s: kept_offsets[%d] < 0", who, b);
+        p.k_off[b] = kept_offsets ? kept_offsets[b] : (int)ksum;
         tok += n_visual[b]; frames += (n_visual[b] + p.tpf - 1) / p.tpf; ksum += k[b];
         if (tok > 0x7fffffffLL / 2) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: too many tokens", who);
     }
@@ -331,15 +334,18 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
         dim3 g1((unsigned)((tok + warps - 1) / warps));
         if (dtype == HIPPO_DTYPE_FP32) select_dots_kernel<float><<<g1, warps * 32, 0, s>>>(p);
         else select_dots_kernel<__nv_bfloat16><<<g1, warps * 32, 0, s>>>(p);
+        count_launches(1);
     }
     if (score_mask & HIPPO_SCORE_SPA) {
         dim3 g2((unsigned)(frames * p.crops_y * p.crops_x));
         if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float><<<g2, 256, 0, s>>>(p);
         else select_spatial_kernel<__nv_bfloat16><<<g2, 256, 0, s>>>(p);
+        count_launches(1);
     }
     const int fuse_threads = ((p.tpf + 31) / 32) * 32;
     select_fuse_kernel<<<(unsigned)frames, fuse_threads, 0, s>>>(p);
-    if (ksum > 0) select_topk_kernel<<<batch, 1024, 0, s>>>(p);
+    count_launches(1);
+    if (ksum > 0) { select_topk_kernel<<<batch, 1024, 0, s>>>(p); count_launches(1); }
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;
 }

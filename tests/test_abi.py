@@ -47,9 +47,9 @@ def test_argument_validation_happens_before_any_launch():
     assert lib.hippo_verify_attention(*args()) == hb.HIPPO_ERR_INVALID_ARG
     n_visual = (ctypes.c_int32 * 1)(100)
     k = (ctypes.c_int32 * 1)(101)
-    assert lib.hippo_select_tokens(1, n_visual, 14, 14, 5, 5, 64, 1, 256, 256, k, 7, 256, 256, 256, 1 << 30, None) == hb.HIPPO_ERR_INVALID_ARG
+    assert lib.hippo_select_tokens(1, n_visual, 14, 14, 5, 5, 64, 1, 256, 256, k, None, 7, 256, 256, 256, 1 << 30, None) == hb.HIPPO_ERR_INVALID_ARG
     k[0] = 10
-    assert lib.hippo_select_tokens(1, n_visual, 14, 14, 6, 6, 64, 1, 256, 256, k, 7, 256, 256, 256, 1 << 30, None) == hb.HIPPO_ERR_UNSUPPORTED_SHAPE
+    assert lib.hippo_select_tokens(1, n_visual, 14, 14, 6, 6, 64, 1, 256, 256, k, None, 7, 256, 256, 256, 1 << 30, None) == hb.HIPPO_ERR_UNSUPPORTED_SHAPE
     assert hb.hippo_select_workspace_bytes([100], 14, 14) >= 256 + 3 * 800
     assert hb.hippo_attention_workspace_bytes(1, 6, 28, 4, 128) > 42 * 130 * 4 * 4
     assert hb.hippo_accept_workspace_bytes(1, 5, 152064) > 0

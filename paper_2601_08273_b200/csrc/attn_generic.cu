@@ -31,7 +31,8 @@ __global__ void __launch_bounds__(kGenThreads) attn_generic_kernel(const AttnPar
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kvl = p.kv_len[b];
-    float *slot = p.partials + ((size_t)(b * p.n_kv_heads + hk) * p.num_splits + split) * ((size_t)R * (D + 2));
+    float *slot = p.partials + ((size_t)(b * p.n_kv_heads + hk) * p.num_splits + split) * slot_float_count(R, D);
+    const int Rp = slot_rows_padded(R);
     if (kvl < p.q_len) return;  // combine writes zeros for such sequences
 
     const T *q = (const T *)p.q;
@@ -90,8 +91,8 @@ __global__ void __launch_bounds__(kGenThreads) attn_generic_kernel(const AttnPar
         }
     }
     __syncthreads();
-    for (int r = tid; r < R; r += kGenThreads) { slot[r] = ms[r]; slot[R + r] = ls[r]; }
-    for (int i = tid; i < R * D; i += kGenThreads) slot[2 * R + i] = Os[i];
+    for (int r = tid; r < R; r += kGenThreads) { slot[r] = ms[r]; slot[Rp + r] = ls[r]; }
+    for (int i = tid; i < R * D; i += kGenThreads) slot[2 * Rp + i] = Os[i];
 }
 
 // One warp per output row (b, t, h): merge the per-split (m, l, O) partials of its (b, kv head).
@@ -111,21 +112,22 @@ __global__ void attn_combine_kernel(const AttnParams p, int n_splits) {
         if (p.lse && lane == 0) p.lse[row] = -INFINITY;
         return;
     }
-    const size_t slot_floats = (size_t)R * (D + 2);
+    const size_t slot_floats = slot_float_count(R, D);
+    const int Rp = slot_rows_padded(R);
     const float *base = p.partials + (size_t)(b * p.n_kv_heads + hk) * n_splits * slot_floats;
     float M = -INFINITY;
     for (int s = 0; s < n_splits; ++s) M = fmaxf(M, base[s * slot_floats + r]);
     float L = 0.f;
     for (int s = 0; s < n_splits; ++s) {
         float m = base[s * slot_floats + r];
-        if (m != -INFINITY) L += base[s * slot_floats + R + r] * expf(m - M);
+        if (m != -INFINITY) L += base[s * slot_floats + Rp + r] * expf(m - M);
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
     for (int d = lane; d < D; d += 32) {
         float acc = 0.f;
         for (int s = 0; s < n_splits; ++s) {
             float m = base[s * slot_floats + r];
-            if (m != -INFINITY) acc = fmaf(base[s * slot_floats + 2 * R + (size_t)r * D + d], expf(m - M), acc);
+            if (m != -INFINITY) acc = fmaf(base[s * slot_floats + 2 * Rp + (size_t)r * D + d], expf(m - M), acc);
         }
         store_from_float(out + d, acc * inv);
     }

@@ -39,6 +39,13 @@ int32_t cuda_fail(cudaError_t e, const char *what);
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// One partial-result slot: m[rows_padded] | l[rows_padded] | O[rows][head_dim] (fp32), rows_padded = rows rounded up
+// to a multiple of 4 so that every part starts on a 16-byte boundary.
+__host__ __device__ inline int slot_rows_padded(int rows) { return (rows + 3) & ~3; }
+__host__ __device__ inline size_t slot_float_count(int rows, int head_dim) {
+    return 2 * (size_t)slot_rows_padded(rows) + (size_t)rows * head_dim;
+}
+
 // Layout of an attention workspace: header | arrival counters | partial slots.
 struct AttnWsLayout {
     size_t counters_off, counters_bytes, partials_off, slot_floats, n_slots, total;
@@ -49,7 +56,7 @@ inline AttnWsLayout attn_ws_layout(int batch, int q_len, int n_q_heads, int n_kv
     L.counters_off = kWsHeaderBytes;
     L.counters_bytes = align_up((size_t)batch * n_kv_heads * sizeof(int32_t), 256);
     L.partials_off = L.counters_off + L.counters_bytes;
-    L.slot_floats = (size_t)rows * (head_dim + 2);
+    L.slot_floats = slot_float_count(rows, head_dim);
     L.n_slots = (size_t)batch * n_kv_heads + kExtraSlots;
     L.total = L.partials_off + align_up(L.n_slots * L.slot_floats * sizeof(float), 256);
     return L;
@@ -66,7 +73,7 @@ struct AttnParams {
     const int32_t *kv_len;
     WsHeader *header;
     int32_t *counters;
-    float *partials;             // n_slots x (rows*(D+2)) floats: m[rows], l[rows], O[rows][D]
+    float *partials;             // n_slots x slot_float_count(rows, D) floats
     int batch, q_len, n_q_heads, n_kv_heads, head_dim, group, rows;
     int n_pages, max_pages_per_seq, max_kv_len;
     int num_splits;

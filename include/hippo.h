@@ -2,7 +2,7 @@
  * hippo.h - C ABI of the B200 (sm_100a) hot path of one HIPPO video speculative-decoding step.
  *
  * Five operations, each a hand-written CUDA kernel family:
- *   hippo_select_tokens     semantic-aware visual-token preservation (Section 4.1, Eq. 3-7 + top-k)
+ *   hippo_select_tokens     semantic-aware visual-token preservation (Section 5.1, Eq. 3-7 + top-k)
  *   hippo_gather_kv         one-time pruning of the draft model's KV cache (Limitations (i))
  *   hippo_draft_attention   draft decode attention over the pruned KV (Section 3.2, drafting phase)
  *   hippo_verify_attention  target verification attention, gamma+1 query tokens (Section 3.2)
@@ -92,7 +92,7 @@ int32_t hippo_workspace_status(const void *workspace, void *stream);
  * once on a fresh workspace before its first use by the attention calls, and after a reported time-out. */
 int32_t hippo_workspace_reset(void *workspace, size_t workspace_bytes, void *stream);
 
-/* ---- selection: Section 4.1 --------------------------------------------------------------------------------- */
+/* ---- selection: Section 5.1 --------------------------------------------------------------------------------- */
 /*
  * For each of `batch` sequences scores its visual tokens and keeps the k best.
  *   Eq. 3-4  s_temp = 1 - mean cosine similarity with the same grid cell in the adjacent frames that contain it

@@ -44,7 +44,7 @@ void oracle_set_threads(int n) {
 }
 
 /* ------------------------------------------------------------------------------------------------
- * Selection: Section 4.1 "Semantic-aware Token Preservation", Eq. 3-7.
+ * Selection: Section 5.1 "Semantic-aware Token Preservation", Eq. 3-7.
  * Tokens are frame-major, row-major inside the frame's grid_h x grid_w patch grid.  The last frame
  * may be partial: it then holds the first (n_visual mod grid_h*grid_w) cells.
  * ---------------------------------------------------------------------------------------------- */
@@ -194,7 +194,7 @@ int oracle_select_scores(int n_visual, int grid_h, int grid_w, int crop_h, int c
     return 0;
 }
 
-/* "retain the top-k visual tokens" (end of Section 4.1): the k best over the whole sequence, ordered by
+/* "retain the top-k visual tokens" (end of Section 5.1): the k best over the whole sequence, ordered by
  * (score descending, index ascending); indices returned ascending.  *kth_score = score of the worst
  * kept token (the threshold). */
 typedef struct { double s; int32_t i; } scored_t;

@@ -1,4 +1,4 @@
-// hippo_select_tokens: semantic-aware visual-token preservation (Section 4.1).
+// hippo_select_tokens: semantic-aware visual-token preservation (Section 5.1).
 //
 //   Eq. 3-4  s_temp(j) = 1 - mean over the adjacent frames that contain j's grid cell of cos(v_j^f, v_j^f')
 //   Eq. 5-6  s_spa(j)  = (1/M) sum_k (S_jk - mu_j)^2 over the M tokens of j's crop, S = cosine Gram matrix, S_jj = 1

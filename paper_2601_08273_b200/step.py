@@ -6,7 +6,7 @@
                           join -> hippo_accept
 
 The draft and the verification kernels run on separate CUDA streams, mirroring the paper's decoupled
-draft/verify overlap (Section 4.2).  This module only allocates device memory through PyTorch, fills it with
+draft/verify overlap (Section 5.2).  This module only allocates device memory through PyTorch, fills it with
 seeded synthetic data and issues the C-ABI calls; every computation is in the CUDA library.  Each layer has its
 own KV buffers, so a pass over the layers streams distinct memory (nothing stays resident in L2 for a cache
 larger than L2).

@@ -187,6 +187,35 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
                      const float *u_resample, int32_t mode, int32_t *n_accepted, int32_t *out_tokens,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * hippo_accept for callers that cannot hand over a workspace.  (No counterpart in the paper: this is a packaging
+ * variant of hippo_accept, same inputs, same outputs, same arithmetic.)
+ *
+ * Who needs it: code that reaches the acceptance step without any means of allocating device memory - a decode
+ * loop whose memory was given in full to an engine's pool at start-up, a plug-in whose host forbids cudaMalloc
+ * because it synchronises the device, glue code that holds only the logits.  The scratch that hippo_accept takes
+ * from its `workspace` argument comes here from an array built into the library image:
+ * HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES bytes of device memory on every GPU that loads libhippo.so, occupied until
+ * the process exits whether or not this function is ever called.
+ *
+ *   - Nothing is allocated or freed, on the device or through any library, by this call.
+ *   - Sizes whose scratch would not fit (hippo_accept_workspace_bytes(batch, gamma, vocab) >
+ *     HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES) are refused with HIPPO_ERR_WORKSPACE_TOO_SMALL before anything is
+ *     launched; hippo_last_error() gives both numbers.  The array covers batch 8, gamma 8 at a 152,064-entry
+ *     vocabulary; larger problems must use hippo_accept.
+ *   - The first call on each device looks up the array's device address (with that device current) and caches
+ *     it.  Make that first call ahead of time, outside any stream capture.
+ *   - All calls on one device share the one array and it keeps whatever the last call left in it.  The kernels
+ *     overwrite every word before reading it, so no clearing is needed, but two calls that may run at the same
+ *     time on the GPU (different streams without an ordering between them) race on it and corrupt each other's
+ *     result.  Order them, or give one of them hippo_accept with its own workspace.
+ */
+#define HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES (256u * 1024u)
+int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vocab, const float *target_logits,
+                             const float *draft_logits, const int32_t *draft_tokens, const float *u_accept,
+                             const float *u_resample, int32_t mode, int32_t *n_accepted, int32_t *out_tokens,
+                             void *stream);
+
 #ifdef __cplusplus
 }
 #endif

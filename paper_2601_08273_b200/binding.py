@@ -71,6 +71,9 @@ lib.hippo_accept_workspace_bytes.restype = _sz
 lib.hippo_accept_workspace_bytes.argtypes = [_i32, _i32, _i32]
 lib.hippo_accept.restype = _i32
 lib.hippo_accept.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp]
+lib.hippo_accept_noalloc.restype = _i32
+lib.hippo_accept_noalloc.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+ACCEPT_NOALLOC_SCRATCH_BYTES = 256 * 1024
 
 
 class HippoError(RuntimeError):
@@ -253,4 +256,25 @@ def hippo_accept(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_
     _check(lib.hippo_accept(B, g, V, _ptr(target_logits), _ptr(draft_logits) if g else None,
                             _ptr(draft_tokens) if g else None, _ptr(u_accept) if g else None, _ptr(u_resample), 0,
                             _ptr(n_accepted), _ptr(out_tokens), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return n_accepted, out_tokens
+
+
+def hippo_accept_noalloc(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                         u_accept: torch.Tensor, u_resample: torch.Tensor, n_accepted: torch.Tensor,
+                         out_tokens: torch.Tensor, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """hippo_accept without a workspace argument, for callers that cannot allocate one (an engine that owns all
+    device memory, a host that forbids cudaMalloc in its decode loop).  The scratch is a fixed array inside the
+    library, shared by every call on the device; the outputs must be passed in because this wrapper allocates
+    nothing either.  Problems needing more than ACCEPT_NOALLOC_SCRATCH_BYTES raise HippoError; calls that may
+    overlap on the GPU must be ordered by the caller."""
+    B, g1, V = target_logits.shape
+    g = g1 - 1
+    for t in (target_logits, draft_logits, u_accept, u_resample):
+        assert t.dtype == torch.float32 and t.is_contiguous()
+    assert draft_tokens.dtype == torch.int32 and draft_tokens.is_contiguous()
+    assert n_accepted.dtype == torch.int32 and n_accepted.numel() >= B
+    assert out_tokens.dtype == torch.int32 and out_tokens.numel() >= B * (g + 1) and out_tokens.is_contiguous()
+    _check(lib.hippo_accept_noalloc(B, g, V, _ptr(target_logits), _ptr(draft_logits) if g else None,
+                                    _ptr(draft_tokens) if g else None, _ptr(u_accept) if g else None,
+                                    _ptr(u_resample), 0, _ptr(n_accepted), _ptr(out_tokens), _stream(stream)))
     return n_accepted, out_tokens

@@ -13,6 +13,8 @@
 //   pick    per sequence: locate the chunk, then the token, where the CDF crosses u * total
 #include <math.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace hippo {
@@ -291,3 +293,79 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
 }
 
 }  // extern "C"
+
+// ---- hippo_accept_noalloc: the same acceptance step for callers that cannot provide a workspace -----------------
+//
+// Some callers have no way to obtain scratch memory at the moment they need to accept a draft: a decode loop whose
+// device memory was handed in full to a serving engine's pool at start-up, a plug-in whose host forbids cudaMalloc
+// (it synchronises the whole device and would stall the draft and verify streams), or glue code that only sees the
+// logits and has no allocator handle at all.  For them the scratch lives in the library image itself: one
+// file-scope device array per GPU that loads libhippo.so, held until the process exits.
+namespace hippo {
+
+constexpr size_t kNoAllocScratchBytes = HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_accept_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void *g_scratch_addr[kMaxDevices] = {nullptr};   // device address of g_accept_scratch, per device ordinal
+static std::mutex g_scratch_mutex;
+
+// In host code `g_accept_scratch` is only a handle for the runtime, not an address a kernel could use.  The real
+// device address differs per GPU and is looked up once per device, with that device current.
+static int32_t noalloc_scratch(void **out) {
+    int dev = -1;
+    HIPPO_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_accept_noalloc: device ordinal %d >= %d", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        HIPPO_CUDA_TRY(cudaGetSymbolAddress((void **)&ptr, g_accept_scratch));
+        if (!ptr || ((uintptr_t)ptr & 255)) return fail(HIPPO_ERR_CUDA, "hippo_accept_noalloc: bad scratch address %p", ptr);
+        g_scratch_addr[dev] = ptr;
+    }
+    *out = g_scratch_addr[dev];
+    return HIPPO_OK;
+}
+
+}  // namespace hippo
+
+extern "C" int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vocab, const float *target_logits,
+                                        const float *draft_logits, const int32_t *draft_tokens, const float *u_accept,
+                                        const float *u_resample, int32_t mode, int32_t *n_accepted, int32_t *out_tokens,
+                                        void *stream) {
+    using namespace hippo;
+    if (batch <= 0 || gamma < 0 || vocab <= 0) return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: bad sizes");
+    if (mode != HIPPO_ACCEPT_SAMPLE) return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept_noalloc: mode %d", mode);
+    if (!target_logits || !u_resample || !n_accepted || !out_tokens)
+        return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: null pointer");
+    if (gamma > 0 && (!draft_logits || !draft_tokens || !u_accept))
+        return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: null draft arrays with gamma > 0");
+    if (gamma > 64 || batch > 65535) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_accept_noalloc: gamma > 64 or batch > 65535");
+    const AcceptWs w = accept_ws(batch, gamma, vocab);
+    if (w.total > kNoAllocScratchBytes)
+        return fail(HIPPO_ERR_WORKSPACE_TOO_SMALL,
+                    "hippo_accept_noalloc: batch %d x gamma %d x vocab %d needs %zu bytes of scratch, the built-in array "
+                    "holds %zu; use hippo_accept with a caller-owned workspace",
+                    batch, gamma, vocab, w.total, kNoAllocScratchBytes);
+    void *scratch = nullptr;
+    const int32_t rc = noalloc_scratch(&scratch);
+    if (rc != HIPPO_OK) return rc;
+    // Every word the kernels read from the scratch is written earlier in the same call (chunk statistics, chunk
+    // weights, the per-sequence record), so nothing has to be cleared although the array keeps the previous
+    // call's contents.
+    AcceptParams p;
+    p.tl = target_logits; p.dl = draft_logits; p.ua = u_accept; p.ur = u_resample; p.x = draft_tokens;
+    p.n_acc = n_accepted; p.out = out_tokens;
+    p.stats = (double2 *)((char *)scratch + w.stats_off);
+    p.wsum = (double *)((char *)scratch + w.wsum_off);
+    p.info = (RowInfo *)((char *)scratch + w.info_off);
+    p.B = batch; p.gamma = gamma; p.V = vocab; p.n_chunks = w.n_chunks;
+    cudaStream_t s = (cudaStream_t)stream;
+    accept_stats_kernel<<<dim3(w.n_chunks, 2 * gamma + 1, batch), kAccThreads, 0, s>>>(p);
+    accept_decide_kernel<<<batch, kAccThreads, (2 * gamma + 1) * 2 * sizeof(double), s>>>(p);
+    accept_wsum_kernel<<<dim3(w.n_chunks, batch), kAccThreads, 0, s>>>(p);
+    accept_pick_kernel<<<batch, kAccThreads, 0, s>>>(p);
+    count_launches(4);
+    HIPPO_CUDA_TRY(cudaGetLastError());
+    return HIPPO_OK;
+}

@@ -13,7 +13,8 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libhippo.so")
+# HIPPO_LIBRARY_PATH selects a libhippo.so built elsewhere (same ABI); default: the in-tree build.
+LIB_PATH = os.environ.get("HIPPO_LIBRARY_PATH") or os.path.join(_PKG, "libhippo.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

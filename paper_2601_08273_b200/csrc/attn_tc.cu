@@ -1,20 +1,30 @@
-// Tensor-core split-KV attention for sm_100a: bf16 K/V pages streamed by TMA, QK^T and PV on tcgen05 with the
+// Tensor-core split-KV attention for sm_100a: bf16 K/V pages streamed by TMA, both contractions on tcgen05 with the
 // accumulators in tensor memory.  Used for the verification pass (gamma+1 query tokens against the full video KV
 // cache) and for the draft decode pass over the pruned cache (Section 3.2).
 //
-// Packing.  All query rows that read one KV head - the q_len tokens times the G = H_q/H_kv heads of its group - are
-// packed as rows r = t*G + g of one M = 128 operand, so every K/V tile is fetched from HBM once per sequence and
-// feeds up to 128 rows of tensor-core work.
+// Operand order.  The path is bound by reading K and V once; the query side is tiny: all query rows that read one
+// KV head - the q_len tokens times the G = H_q/H_kv heads of its group, R = q_len*G <= 128 rows, padded to
+// Rp = multiple of 16 - are packed as row r = t*G + g.  A tile is 128 keys (two pages).  The keys go on the M
+// dimension of the MMA and the packed rows on N, so no tensor-core or softmax lane is spent on padding rows:
+//     S^T [128 keys x Rp] = K_tile [128 x D] . Q^T        (A = K pages as TMA wrote them, B = Q in shared memory)
+//     O^T [D x Rp]       += V_tile^T [D x 128] . P^T       (A = V pages as TMA wrote them, read M-major; B = P^T)
+// One tcgen05.mma costs about 60 cycles whatever its size below N = 128, so the tile is shaped to need few of
+// them: 8 + 8 per 64 KB of K/V.  A softmax thread owns one key and walks the Rp rows; its partial row sums
+// accumulate in tensor memory next to S^T and are reduced over the keys once per segment.  The only cross-thread
+// traffic of a tile is one OR-reduction: "did any score rise more than 2^8 above the row's reference maximum?".
+// If not (the common case after the first tile) the stale reference is kept; otherwise the exact row maxima are
+// recomputed and O^T and the partial sums are rescaled in tensor memory.
 //
-// Work split.  The 64-key tiles of all (sequence, kv head) units form one flat list that is cut into gridDim.x equal
+// Work split.  The tiles of all (sequence, kv head) units form one flat list that is cut into gridDim.x equal
 // contiguous ranges (persistent CTAs, one per SM).  A CTA walks its range unit by unit ("segments"); for each
 // segment it produces either the final output (it owns the whole unit) or a partial (m, l, O) in slot unit+cta of
 // the workspace, which the combine kernel merges.
 //
-// CTA = 6 warps:  warp 0 TMA producer (ring of kStages K+V tiles, full/empty mbarriers)
-//                 warp 1 tcgen05.mma issuer and TMEM owner:  S[j] = Q K_i^T  (double buffered),  O += P_i V_i
-//                 warps 2-5: one thread per packed row: S -> registers, online softmax in base 2 with lazy
-//                 rescaling of O, P -> shared memory (bf16, 128B swizzle), epilogue.
+// CTA = 10 warps: warp 0 TMA producer: ring of 2-page slots, alternately K and V of a tile, full/empty mbarriers;
+//                        a K slot is released as soon as QK^T has read it
+//                 warp 1 tcgen05.mma issuer and TMEM owner; S^T double buffered, PV trails QK by one tile
+//                 warps 2-9 softmax / rescale / epilogue: warps w and w+4 share a quarter of the tensor-memory
+//                        lanes and split the packed rows in alternating groups of 16
 // Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA records HIPPO_ERR_TIMEOUT in the
 // workspace header, drains its own copies, frees its tensor memory and exits.
 #include <cuda.h>
@@ -24,26 +34,16 @@
 
 namespace hippo {
 
-constexpr int kTcThreads = 192;
-constexpr int kBlockN = 64;            // keys per tile = one KV page
-constexpr int kBlockM = 128;           // packed rows (padded)
+constexpr int kTcThreads = 320;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kBlockN = 128;           // keys per tile = two KV pages
+constexpr int kMaxRows = 128;          // packed rows (padded)
+constexpr int kMaxSlots = 12;
 constexpr int kTcMaxBatch = 256;       // per-sequence tile prefix lives in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;              // lazy rescale: only when the running max grows by > 2^8
+constexpr float kRescaleThreshold = 8.0f;              // lazy rescale: only when a score exceeds the reference by > 2^8
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
-
-template <int D> struct TcCfg {
-    static constexpr int kChunks = D / 64;                       // 64-column (128-byte) swizzle chunks per row
-    static constexpr int kQBytes = kBlockM * D * 2;
-    static constexpr int kPBytes = kBlockM * kBlockN * 2;         // one P buffer
-    static constexpr int kTileBytes = kBlockN * D * 2;            // one K or V tile
-    static constexpr int kStageBytes = 2 * kTileBytes;
-    static constexpr int kStages = D == 128 ? 5 : 8;
-    static constexpr int kDataBytes = kQBytes + 2 * kPBytes + kStages * kStageBytes;
-    static constexpr int kTmemCols = 256;                         // S0 | S1 | O
-    static constexpr int kColS = 0, kColO = 128;
-};
 
 // ---- PTX wrappers -------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -81,24 +81,19 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+// 16 consecutive columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
     uint32_t *r = reinterpret_cast<uint32_t *>(v);
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-                   "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-                   "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-                   "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                   "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
                  : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *v) {
     const uint32_t *r = reinterpret_cast<const uint32_t *>(v);
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
                  ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-                   "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-                   "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-                   "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                   "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
                  : "memory");
 }
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -106,17 +101,31 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float warp_max(float x) {
+    float y;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor, 128-byte swizzle, Blackwell version field.  Offsets in bytes.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-           (1ull << 46) | (2ull << 61);
+// Barrier 1 is private to the 256 softmax threads.
+__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ bool softmax_bar_or(bool pred) {
+    uint32_t out;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(out) : "r"((uint32_t)pred) : "memory");
+    return out != 0;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major, B K-major or MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
+
+// Shared-memory matrix descriptor (Blackwell version field set).  Offsets in bytes.  swizzle: 0 none, 2 = 128 bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | ((uint64_t)swizzle << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32.  *_mn: operand is contiguous along M (A) / N (B) instead of K.
+__device__ __forceinline__ uint32_t instr_desc(int m, int n, bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // ---- work partition (shared by the main and the combine kernel) ---------------------------------------------------
@@ -131,9 +140,14 @@ __device__ __forceinline__ int seq_tiles(int kvl, int q_len) { return kvl < q_le
 
 // ---- shared control block -------------------------------------------------------------------------------------------
 struct TcShared {
-    unsigned long long full[8], empty[8], s_full[2], s_free[2], p_full[2], pv_done[2], q_full, q_free, drain;
+    unsigned long long full[kMaxSlots], empty[kMaxSlots], s_full[2], s_free[2], p_full[2], pv_done[2], q_full, q_free, drain;
     uint32_t tmem_base;
     volatile int abort;
+    float mneg[kMaxRows];       // minus the reference maximum of each packed row, log2 domain (+inf: nothing seen yet)
+    float fscale[kMaxRows];     // rescale factors of a slow path; row sums in the epilogue
+    float wpart[4][kMaxRows];   // per-warp tile maxima (slow path) / per-warp row sums (epilogue)
+    int limit[kMaxRows];        // last visible key of each packed row
+    int rowoff[kMaxRows];       // (b*q_len + t)*H_q + h of each packed row, -1 for padding rows
     int tile_prefix[kTcMaxBatch + 1];  // only [0, batch] used
 };
 
@@ -159,19 +173,43 @@ struct Waiter {
     }
 };
 
-template <int D> constexpr int tc_smem_bytes() { return TcCfg<D>::kDataBytes + 1024 /* alignment */ + (int)sizeof(TcShared); }
-static_assert(tc_smem_bytes<128>() <= 227 * 1024, "shared memory budget");
+// Position in the slot ring: slot index and the parity of its current use.
+struct RingPos {
+    int slot;
+    uint32_t phase;
+    __device__ __forceinline__ void advance(int n_slots) {
+        if (++slot == n_slots) { slot = 0; phase ^= 1; }
+    }
+};
+
+struct TcSmemPlan { int q_bytes, p_bytes, fixed, slots, total; };
+// Shared-memory carve-up: [ring of 2-page slots | Q | P^T x2 | control], ring depth = whatever fits.
+static TcSmemPlan tc_smem_plan(int D, int Rp) {
+    TcSmemPlan s;
+    s.q_bytes = Rp * D * 2;
+    s.p_bytes = Rp * kBlockN * 2;
+    s.fixed = s.q_bytes + 2 * s.p_bytes + (int)((sizeof(TcShared) + 127) & ~(size_t)127);
+    const int slot = kBlockN * D * 2;
+    int n = (227 * 1024 - 1024 - s.fixed) / slot;
+    s.slots = n > kMaxSlots ? kMaxSlots : n;
+    s.total = 1024 + s.fixed + s.slots * slot;
+    return s;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
-attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
-    using C = TcCfg<D>;
+attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+               const int Rp, const int n_slots, const int tmem_cols) {
+    constexpr int kChunks = D / 64;                     // 64-column (128-byte) swizzle chunks per row
+    constexpr int kPageBytes = kPageSize * D * 2;       // K or V of one page and head
+    constexpr int kSlotBytes = 2 * kPageBytes;          // K or V of one tile
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t *q_s = base;                                    // [kChunks][128 rows][128 B]
-    uint8_t *p_s = q_s + C::kQBytes;                        // [2][128 rows][128 B]
-    uint8_t *kv_s = p_s + 2 * C::kPBytes;                   // [kStages][K: kChunks x 8 KB | V: kChunks x 8 KB]
-    TcShared *sh = (TcShared *)(kv_s + C::kStages * C::kStageBytes);
+    uint8_t *ring = base;                                   // [n_slots] K: [chunk][page][64 rows][128 B]; V: [page][chunk][64][128 B]
+    uint8_t *q_s = ring + n_slots * kSlotBytes;             // [kChunks][Rp rows][128 B], 128B swizzle
+    uint8_t *p_s = q_s + Rp * D * 2;                        // [2][Rp/8][128 keys][8 rows] bf16 (no swizzle, row-contiguous)
+    TcShared *sh = (TcShared *)(p_s + 2 * Rp * kBlockN * 2);
+    const int p_bytes = Rp * kBlockN * 2;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = p.rows, G = p.group, Hkv = p.n_kv_heads, B = p.batch;
@@ -179,14 +217,14 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
 
     // ---- set-up: barriers, tile prefix, tensor memory
     if (tid == 0) {
-        for (int s = 0; s < C::kStages; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
+        for (int s = 0; s < n_slots; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
         for (int j = 0; j < 2; ++j) {
             mbar_init(smem_u32(&sh->s_full[j]), 1);
-            mbar_init(smem_u32(&sh->s_free[j]), 128);
-            mbar_init(smem_u32(&sh->p_full[j]), 128);
+            mbar_init(smem_u32(&sh->s_free[j]), kSoftmaxThreads);
+            mbar_init(smem_u32(&sh->p_full[j]), kSoftmaxThreads);
             mbar_init(smem_u32(&sh->pv_done[j]), 1);
         }
-        mbar_init(smem_u32(&sh->q_full), 128);
+        mbar_init(smem_u32(&sh->q_full), kSoftmaxThreads);
         mbar_init(smem_u32(&sh->q_free), 1);
         mbar_init(smem_u32(&sh->drain), 1);
         sh->abort = 0;
@@ -195,14 +233,19 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         sh->tile_prefix[B] = acc;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (tid == 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&v_map) : "memory");
+    }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
+    const uint32_t col_s = 0, col_o = 2 * Rp, col_l = 3 * Rp;   // S^T[0] | S^T[1] | O^T | partial row sums, Rp columns each
 
     Partition part;
     part.total = (long long)sh->tile_prefix[B] * Hkv;
@@ -210,18 +253,16 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     const long long t_begin = part.total > 0 ? part.start_of(blockIdx.x) : 0;
     const long long t_end = part.total > 0 ? part.start_of(blockIdx.x + 1) : 0;
 
-    // Segment iteration state shared by all roles: each role walks the same list of segments.
-    // A segment = (b, hk, first tile, tile count, final?) derived from the flat range [t_begin, t_end).
+    // Every role walks the same list of segments.  A segment = (b, hk, first tile, tile count) taken from the flat
+    // range [t_begin, t_end); order is unit-major: all tiles of (b, hk=0), then (b, hk=1), ...
     auto locate = [&](long long t, int &b, int &hk, int &tile) {
-        // unit-major order: all tiles of (b, hk=0), then (b, hk=1), ...
         int lo = 0, hi = B;  // largest b with Hkv * prefix[b] <= t
         while (hi - lo > 1) {
             int mid = (lo + hi) >> 1;
             if ((long long)sh->tile_prefix[mid] * Hkv <= t) lo = mid; else hi = mid;
         }
-        // skip sequences with zero tiles that share the same prefix
         b = lo;
-        while (b + 1 < B && (long long)sh->tile_prefix[b + 1] * Hkv <= t) ++b;
+        while (b + 1 < B && (long long)sh->tile_prefix[b + 1] * Hkv <= t) ++b;   // skip sequences without tiles
         const int nt = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
         const long long off = t - (long long)sh->tile_prefix[b] * Hkv;
         hk = (int)(off / nt);
@@ -231,7 +272,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            uint32_t it = 0;
+            RingPos rp{0, 0};
+            uint32_t issued = 0;
             long long t = t_begin;
             bool ok = true;
             while (ok && t < t_end) {
@@ -239,48 +281,70 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 locate(t, b, hk, tile);
                 const int nt = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
                 const int n = (int)min((long long)(nt - tile), t_end - t);
-                for (int i = 0; i < n && ok; ++i, ++it) {
-                    const int s = it % C::kStages;
-                    ok = W.wait(&sh->empty[s], ((it / C::kStages) & 1) ^ 1, 1);
-                    if (!ok) break;
-                    const int pid = page_of(p.page_table, p.max_pages_per_seq, b, tile + i);
-                    const int row = (pid * Hkv + hk) * kPageSize;
-                    const uint32_t bar = smem_u32(&sh->full[s]);
-                    mbar_expect_tx(bar, C::kStageBytes);
-                    const uint32_t dst = smem_u32(kv_s + s * C::kStageBytes);
+                const int n_pages_seq = (p.kv_len[b] + kPageSize - 1) / kPageSize;
+                for (int i = 0; i < n && ok; ++i) {
+                    const int pg0 = 2 * (tile + i);
+                    const int np = min(2, n_pages_seq - pg0);        // the last tile of a sequence may hold one page
+                    int row[2];
+                    for (int q = 0; q < np; ++q)
+                        row[q] = (page_of(p.page_table, p.max_pages_per_seq, b, pg0 + q) * Hkv + hk) * kPageSize;
+                    // K of the tile, then V of the tile
+                    for (int kv = 0; kv < 2 && ok; ++kv, rp.advance(n_slots), ++issued) {
+                        ok = W.wait(&sh->empty[rp.slot], rp.phase ^ 1, 1);
+                        if (!ok) break;
+                        const uint32_t bar = smem_u32(&sh->full[rp.slot]);
+                        mbar_expect_tx(bar, np * kPageBytes);
+                        const uint32_t dst = smem_u32(ring + rp.slot * kSlotBytes);
+                        for (int q = 0; q < np; ++q) {
 #pragma unroll
-                    for (int c = 0; c < C::kChunks; ++c) tma_load_2d(dst + c * 8192, &k_map, c * 64, row, bar);
-#pragma unroll
-                    for (int c = 0; c < C::kChunks; ++c) tma_load_2d(dst + C::kTileBytes + c * 8192, &v_map, c * 64, row, bar);
+                            for (int c = 0; c < kChunks; ++c) {
+                                if (kv == 0) tma_load_2d(dst + c * (2 * 8192) + q * 8192, &k_map, c * 64, row[q], bar);
+                                else tma_load_2d(dst + q * kPageBytes + c * 8192, &v_map, c * 64, row[q], bar);
+                            }
+                        }
+                    }
                 }
                 t += n;
             }
             // drain: every load that was issued must have landed before the CTA may exit
-            const uint32_t issued = it;
-            for (uint32_t k = (issued > (uint32_t)C::kStages ? issued - C::kStages : 0); k < issued; ++k)
-                W.wait(&sh->full[k % C::kStages], (k / C::kStages) & 1, 2);
+            const int back = issued < (uint32_t)n_slots ? (int)issued : n_slots;
+            for (int k = 0; k < back; ++k) {
+                // step the ring position back by one
+                if (rp.slot == 0) { rp.slot = n_slots - 1; rp.phase ^= 1; } else --rp.slot;
+                W.wait(&sh->full[rp.slot], rp.phase, 2);
+            }
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc(kBlockN, false);
-            constexpr uint32_t idesc_pv = instr_desc(D, true);
+            const uint32_t idesc_qk = instr_desc(kBlockN, Rp, false, false);   // S^T: A = K (K-major), B = Q (K-major)
+            const uint32_t idesc_pv = instr_desc(D, Rp, true, true);           // O^T: A = V (M-major), B = P^T (N-major)
+            // descriptors of the operands at offset 0; an operand at byte offset x adds x >> 4 to the address field
+            const uint64_t kdesc0 = smem_desc(smem_u32(ring), 16, 1024, 2);
+            const uint64_t vdesc0 = smem_desc(smem_u32(ring), 8192, 1024, 2);
+            const uint64_t qdesc0 = smem_desc(smem_u32(q_s), 16, 1024, 2);
+            const uint64_t pdesc0 = smem_desc(smem_u32(p_s), 128, kBlockN * 16, 0);
+            const uint32_t q_chunk16 = (uint32_t)(Rp * 128) >> 4;
+            RingPos rk{0, 0};            // slot of the next tile's K
+            RingPos rv{1 % n_slots, (uint32_t)(n_slots == 1)};   // slot of the next PV's V (K and V alternate in the ring)
             uint32_t it = 0, seg = 0;
             long long t = t_begin;
             bool ok = true;
-            // issues O += P_i V_i for global tile counter `k` (stage and buffers derive from k)
+            // O^T += V_k^T P_k^T for the CTA's tile number k
             auto issue_pv = [&](uint32_t k, bool first_of_segment) -> bool {
-                const int j = k & 1, s = k % C::kStages;
+                const int j = k & 1;
+                if (!W.wait(&sh->full[rv.slot], rv.phase, 15)) return false;
                 if (!W.wait(&sh->p_full[j], (k >> 1) & 1, 3)) return false;
                 tc_fence_after();
-                const uint32_t pa = smem_u32(p_s + j * C::kPBytes);
-                const uint32_t va = smem_u32(kv_s + s * C::kStageBytes + C::kTileBytes);
+                const uint64_t pd = pdesc0 + (uint64_t)((uint32_t)(j * p_bytes) >> 4);
+                const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)(rv.slot * kSlotBytes) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < kBlockN / 16; ++ks)
-                    tc_mma(tmem + C::kColO, smem_desc(pa + ks * 32, 16, 1024), smem_desc(va + ks * 2048, 8192, 1024), idesc_pv,
-                           (first_of_segment && ks == 0) ? 0u : 1u);
+                    tc_mma(tmem + col_o, vd + (uint64_t)(((ks >> 2) * kPageBytes + (ks & 3) * 2048) >> 4), pd + (uint64_t)((ks * 256) >> 4),
+                           idesc_pv, (first_of_segment && ks == 0) ? 0u : 1u);
                 tc_commit(smem_u32(&sh->pv_done[j]));
-                tc_commit(smem_u32(&sh->empty[s]));
+                tc_commit(smem_u32(&sh->empty[rv.slot]));
+                rv.advance(n_slots); rv.advance(n_slots);
                 return true;
             };
             while (ok && t < t_end) {
@@ -291,24 +355,26 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 ok = W.wait(&sh->q_full, seg & 1, 4);  // Q of this segment is in shared memory
                 const uint32_t it0 = it;
                 for (int i = 0; i < n && ok; ++i, ++it) {
-                    const int j = it & 1, s = it % C::kStages;
-                    ok = W.wait(&sh->full[s], (it / C::kStages) & 1, 5);
+                    const int j = it & 1;
+                    ok = W.wait(&sh->full[rk.slot], rk.phase, 5);
                     if (!ok) break;
-                    // S buffer j was last read by the softmax of tile it-2
+                    // S^T buffer j was last read by the softmax of tile it-2
                     if (it >= 2) { ok = W.wait(&sh->s_free[j], ((it - 2) >> 1) & 1, 14); if (!ok) break; }
                     tc_fence_after();
-                    const uint32_t qa = smem_u32(q_s), ka = smem_u32(kv_s + s * C::kStageBytes);
+                    const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)(rk.slot * kSlotBytes) >> 4);
 #pragma unroll
-                    for (int c = 0; c < C::kChunks; ++c)
+                    for (int c = 0; c < kChunks; ++c)
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            tc_mma(tmem + C::kColS + j * kBlockN, smem_desc(qa + c * 16384 + ks * 32, 16, 1024),
-                                   smem_desc(ka + c * 8192 + ks * 32, 16, 1024), idesc_qk, (c | ks) ? 1u : 0u);
+                            tc_mma(tmem + col_s + j * Rp, kd + (uint64_t)((c * (2 * 8192) + ks * 32) >> 4),
+                                   qdesc0 + (uint64_t)(c * q_chunk16 + ks * 2), idesc_qk, (c | ks) ? 1u : 0u);
                     tc_commit(smem_u32(&sh->s_full[j]));
-                    if (i == n - 1) tc_commit(smem_u32(&sh->q_free));  // last QK of the segment: Q may be replaced
-                    if (i >= 2) ok = issue_pv(it - 2, it - 2 == it0);    // PV trails QK by two tiles
+                    tc_commit(smem_u32(&sh->empty[rk.slot]));            // K is not needed again
+                    if (i == n - 1) tc_commit(smem_u32(&sh->q_free));    // last QK of the segment: Q may be replaced
+                    rk.advance(n_slots); rk.advance(n_slots);
+                    if (i >= 1) ok = issue_pv(it - 1, it - 1 == it0);    // PV trails QK by one tile
                 }
-                for (uint32_t k = (n >= 2 ? it - 2 : it0); ok && k < it; ++k) ok = issue_pv(k, k == it0);
+                if (ok && n >= 1) ok = issue_pv(it - 1, it - 1 == it0);
                 t += n;
                 ++seg;
             }
@@ -317,176 +383,257 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             W.wait(&sh->drain, 0, 6);
         }
     } else {
-        // ================= softmax / epilogue: one thread per packed row =================
-        const int quarter = warp & 3;                 // TMEM lanes this warp may access: 32*quarter .. +31
-        const int r = quarter * 32 + lane;            // packed row
-        const bool warp_active = quarter * 32 < R;
-        const bool row_active = r < R;
+        // ================= softmax / rescale / epilogue =================
+        // Tensor memory: a warp reaches lanes 32*(warp%4)..+31.  S^T and the partial row sums keep key 32*q + l of
+        // the tile on lane 32*q + l; O^T keeps output dimension d on lane d (D = 128) or on lane 32*(d/16) + d%16
+        // (D = 64, an M = 64 accumulator).  Control flow below is uniform over the 256 threads between named
+        // barriers: a failed wait is remembered in `ok` and acted upon only right after the per-tile reduction.
+        const int st = tid - 64;                      // 0..255
+        const int quarter = warp & 3;
+        const int c_first = ((warp - 2) >> 2) * 16;   // this warp's row groups: c_first, c_first + 32, ...
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const int kk = quarter * 32 + lane;           // key inside the tile
+        const bool d_active = (D == 128) || lane < 16;
+        const int d = (D == 128) ? quarter * 32 + lane : quarter * 16 + lane;
         const float sl2 = p.scale * kLog2e;
-        const int t_row = r / G, g_row = r % G;
+        RingPos rv{1 % n_slots, (uint32_t)(n_slots == 1)};   // slot of the current tile's V
         uint32_t it = 0, seg = 0;
         long long t = t_begin;
         bool ok = true;
-        while (ok && t < t_end) {
+        while (t < t_end) {
             int b, hk, tile;
             locate(t, b, hk, tile);
             const int nt = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
             const int n = (int)min((long long)(nt - tile), t_end - t);
             const int kvl = p.kv_len[b];
             const bool whole_unit = (tile == 0 && n == nt);
-            // ---- Q of this segment -> shared memory (swizzled K-major), after the previous segment's QK MMAs are done
-            if (seg > 0) ok = W.wait(&sh->q_free, (seg - 1) & 1, 7);
-            if (!ok) break;
-            {
-                const __nv_bfloat16 *qg = (const __nv_bfloat16 *)p.q + (((size_t)b * p.q_len + t_row) * p.n_q_heads + hk * G + g_row) * D;
-#pragma unroll
-                for (int c = 0; c < D / 8; ++c) {
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (row_active) v = __ldg(reinterpret_cast<const uint4 *>(qg) + c);
-                    *reinterpret_cast<uint4 *>(q_s + (c >> 3) * 16384 + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+            // ---- per-segment tables and Q -> shared memory (after the previous segment's QK MMAs are done)
+            if (seg > 0) ok = W.wait(&sh->q_free, (seg - 1) & 1, 7) && ok;
+            if (st < Rp) {
+                if (st < R) {
+                    const int tq = st / G, g = st % G;
+                    sh->limit[st] = kvl - p.q_len + tq;
+                    sh->rowoff[st] = (b * p.q_len + tq) * p.n_q_heads + hk * G + g;
+                } else {
+                    sh->limit[st] = 0x7fffffff;
+                    sh->rowoff[st] = -1;
                 }
-                fence_proxy_async();
-                mbar_arrive(smem_u32(&sh->q_full));
+                sh->mneg[st] = INFINITY;
             }
-            const int limit = kvl - p.q_len + t_row;   // last visible key of this row
-            float m_ref = -INFINITY, l_sum = 0.f;
+            softmax_bar_sync();
+            for (int x = st; x < Rp * (D / 8); x += kSoftmaxThreads) {
+                const int r = x / (D / 8), c = x % (D / 8);
+                uint4 v = make_uint4(0, 0, 0, 0);
+                const int ro = sh->rowoff[r];
+                if (ro >= 0) v = __ldg(reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)p.q + (size_t)ro * D) + c);
+                *reinterpret_cast<uint4 *>(q_s + (c >> 3) * (Rp * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+            }
+            fence_proxy_async();
+            mbar_arrive(smem_u32(&sh->q_full));
+
             const uint32_t it0 = it;
-            for (int i = 0; i < n && ok; ++i, ++it) {
-                const int j = it & 1, s = it % C::kStages;
+            bool aborted = false;
+            for (int i = 0; i < n; ++i, ++it, rv.advance(n_slots), rv.advance(n_slots)) {
+                const int j = it & 1;
                 const int key0 = (tile + i) * kBlockN;
+                const int key = key0 + kk;
                 const bool tail = key0 + kBlockN > kvl - p.q_len + 1;  // some row needs masking in this tile
+                const uint32_t s_addr = tmem + lane_addr + col_s + j * Rp;
                 if (key0 + kBlockN > kvl) {
-                    // rows of V past the end of the sequence may hold anything: zero them (0 * NaN would poison O)
-                    ok = W.wait(&sh->full[s], (it / C::kStages) & 1, 8);
-                    if (!ok) break;
-                    uint8_t *vs = kv_s + s * C::kStageBytes + C::kTileBytes;
+                    // rows of V past the end of the sequence may hold anything (also a whole missing second page):
+                    // zero them, 0 * NaN would poison O
+                    ok = W.wait(&sh->full[rv.slot], rv.phase, 8) && ok;
+                    uint8_t *vs = ring + rv.slot * kSlotBytes;
                     const int first_bad = kvl - key0;
-                    for (int x = (tid - 64); x < (kBlockN - first_bad) * C::kChunks * 8; x += 128) {
-                        const int row = first_bad + x / (C::kChunks * 8), rem = x % (C::kChunks * 8);
-                        *reinterpret_cast<uint4 *>(vs + (rem >> 3) * 8192 + row * 128 + ((rem & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    for (int x = st; x < (kBlockN - first_bad) * kChunks * 8; x += kSoftmaxThreads) {
+                        const int row = first_bad + x / (kChunks * 8), rem = x % (kChunks * 8);
+                        *reinterpret_cast<uint4 *>(vs + (row >> 6) * kPageBytes + (rem >> 3) * 8192 + (row & 63) * 128 + ((rem & 7) << 4)) =
+                            make_uint4(0, 0, 0, 0);
                     }
                     fence_proxy_async();
                 }
-                ok = W.wait(&sh->s_full[j], (it >> 1) & 1, 9);
-                if (!ok) break;
+                ok = W.wait(&sh->s_full[j], (it >> 1) & 1, 9) && ok;
                 tc_fence_after();
-                float sv[kBlockN];
-                if (warp_active) {
-                    tmem_ld32(tmem + lane_addr + C::kColS + j * kBlockN, sv);
-                    tmem_ld32(tmem + lane_addr + C::kColS + j * kBlockN + 32, sv + 32);
-                    tmem_wait_ld();
-                    tc_fence_before();
-                    mbar_arrive(smem_u32(&sh->s_free[j]));   // S buffer may be overwritten by QK of tile it+2
-                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                // ---- pass 1: does any visible score exceed its row's reference by more than the threshold?
+                // (branch-free inside; the masked variant runs only for the last tiles of a sequence)
+                float excess = -INFINITY;
+                if (!tail) {
+                    for (int c = c_first; c < Rp; c += 32) {
+                        float sv[16];
+                        tmem_ld16(s_addr + c, sv);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < kBlockN; ++c) {
-                        float x = sv[c] * sl2;
-                        if (tail && key0 + c > limit) x = -INFINITY;
-                        sv[c] = x;
-                        mx4[c & 3] = fmaxf(mx4[c & 3], x);
-                    }
-                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                    // lazy rescale of the running output: only when the maximum moved by more than the threshold
-                    bool need = (m_ref == -INFINITY) ? false : (mx > m_ref + kRescaleThreshold);
-                    if (m_ref == -INFINITY && mx != -INFINITY) m_ref = mx;   // first visible keys: adopt, O is still empty
-                    if (__any_sync(0xffffffffu, need)) {
-                        // O holds tiles it0..it-1: wait until PV of tile it-1 has been accumulated
-                        if (it > it0) {
-                            ok = W.wait(&sh->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1, 10);
-                            if (!ok) break;
-                            tc_fence_after();
-                            const float f = need ? exp2f(m_ref - mx) : 1.f;
-                            float ov[32];
-#pragma unroll
-                            for (int c = 0; c < D / 32; ++c) {
-                                tmem_ld32(tmem + lane_addr + C::kColO + c * 32, ov);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int e = 0; e < 32; ++e) ov[e] *= f;
-                                tmem_st32(tmem + lane_addr + C::kColO + c * 32, ov);
-                            }
-                            tmem_wait_st();
-                            if (need) { l_sum *= f; m_ref = mx; }
-                        } else if (need) {
-                            l_sum *= exp2f(m_ref - mx);
-                            m_ref = mx;
+                        for (int e4 = 0; e4 < 4; ++e4) {
+                            const float4 mn = *reinterpret_cast<const float4 *>(&sh->mneg[c + 4 * e4]);
+                            excess = fmaxf(excess, fmaxf(fmaxf(fmaf(sv[4 * e4], sl2, mn.x), fmaf(sv[4 * e4 + 1], sl2, mn.y)),
+                                                         fmaxf(fmaf(sv[4 * e4 + 2], sl2, mn.z), fmaf(sv[4 * e4 + 3], sl2, mn.w))));
                         }
                     }
-                    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                    // P buffer j was last read by PV of tile it-2
-                    if (it >= 2) { ok = W.wait(&sh->pv_done[j], ((it - 2) >> 1) & 1, 11); if (!ok) break; }
-                    uint8_t *prow = p_s + j * C::kPBytes + r * 128;
-                    float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                    for (int c = 0; c < kBlockN / 8; ++c) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float a = ex2_approx(sv[c * 8 + 2 * e] - m_use), bb = ex2_approx(sv[c * 8 + 2 * e + 1] - m_use);
-                            ls4[e] += a + bb;
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(a, bb);
-                            w[e] = *reinterpret_cast<uint32_t *>(&h2);
-                        }
-                        *reinterpret_cast<uint4 *>(prow + ((c ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                    l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
                 } else {
-                    mbar_arrive(smem_u32(&sh->s_free[j]));
-                    if (it >= 2) { ok = W.wait(&sh->pv_done[j], ((it - 2) >> 1) & 1, 12); if (!ok) break; }
+                    for (int c = c_first; c < Rp; c += 32) {
+                        float sv[16];
+                        tmem_ld16(s_addr + c, sv);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e4 = 0; e4 < 4; ++e4) {
+                            const float4 mn = *reinterpret_cast<const float4 *>(&sh->mneg[c + 4 * e4]);
+                            const int4 lm = *reinterpret_cast<const int4 *>(&sh->limit[c + 4 * e4]);
+                            const float x0 = fmaf(sv[4 * e4], sl2, mn.x), x1 = fmaf(sv[4 * e4 + 1], sl2, mn.y);
+                            const float x2 = fmaf(sv[4 * e4 + 2], sl2, mn.z), x3 = fmaf(sv[4 * e4 + 3], sl2, mn.w);
+                            excess = fmaxf(excess, fmaxf(fmaxf(key <= lm.x ? x0 : -INFINITY, key <= lm.y ? x1 : -INFINITY),
+                                                         fmaxf(key <= lm.z ? x2 : -INFINITY, key <= lm.w ? x3 : -INFINITY)));
+                        }
+                    }
                 }
-                fence_proxy_async();
+                // a NaN excess (inf - inf on a row that has seen nothing) must count as growth
+                const bool grow = !(excess <= kRescaleThreshold);
+                const bool any_grow = softmax_bar_or(grow || !ok);
+                if (sh->abort) { aborted = true; break; }
+                if (any_grow) {
+                    // ---- exact tile maxima per row, new references, rescale of what has been accumulated
+                    for (int c = c_first; c < Rp; c += 32) {
+                        float sv[16];
+                        tmem_ld16(s_addr + c, sv);
+                        tmem_wait_ld();
+                        float mine = -INFINITY;
+                        if (tail) {   // uniform over the CTA
+#pragma unroll
+                            for (int e4 = 0; e4 < 4; ++e4) {
+                                const int4 lm = *reinterpret_cast<const int4 *>(&sh->limit[c + 4 * e4]);
+                                sv[4 * e4] = key <= lm.x ? sv[4 * e4] : -INFINITY;
+                                sv[4 * e4 + 1] = key <= lm.y ? sv[4 * e4 + 1] : -INFINITY;
+                                sv[4 * e4 + 2] = key <= lm.z ? sv[4 * e4 + 2] : -INFINITY;
+                                sv[4 * e4 + 3] = key <= lm.w ? sv[4 * e4 + 3] : -INFINITY;
+                            }
+                        }
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float y = warp_max(sv[e] * sl2);
+                            mine = (lane == e) ? y : mine;
+                        }
+                        if (lane < 16) sh->wpart[quarter][c + lane] = mine;
+                    }
+                    softmax_bar_sync();
+                    if (st < Rp) {
+                        const float m_old = -sh->mneg[st];
+                        const float tm = fmaxf(fmaxf(sh->wpart[0][st], sh->wpart[1][st]), fmaxf(sh->wpart[2][st], sh->wpart[3][st]));
+                        const float m_new = fmaxf(m_old, tm);
+                        float f = 1.f;
+                        if (m_new != -INFINITY) {
+                            f = (m_old == -INFINITY) ? 0.f : exp2f(m_old - m_new);
+                            sh->mneg[st] = -m_new;
+                        }
+                        sh->fscale[st] = f;
+                    }
+                    softmax_bar_sync();
+                    if (it > it0) {
+                        // O^T and the partial sums hold tiles it0..it-1: wait until PV of tile it-1 has been accumulated
+                        ok = W.wait(&sh->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1, 10) && ok;
+                        tc_fence_after();
+                        for (int c = c_first; c < Rp; c += 32) {
+                            float ov[16], lv[16];
+                            tmem_ld16(tmem + lane_addr + col_o + c, ov);
+                            tmem_ld16(tmem + lane_addr + col_l + c, lv);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) { const float f = sh->fscale[c + e]; ov[e] *= f; lv[e] *= f; }
+                            tmem_st16(tmem + lane_addr + col_o + c, ov);
+                            tmem_st16(tmem + lane_addr + col_l + c, lv);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                // ---- pass 2: P^T = 2^(s*scale*log2e - reference) as bf16, row-contiguous per key; partial row sums
+                // P^T buffer j was last read by PV of tile it-2
+                if (it >= 2) ok = W.wait(&sh->pv_done[j], ((it - 2) >> 1) & 1, 11) && ok;
+                uint8_t *pk = p_s + j * p_bytes + kk * 16;
+                const bool first_tile = it == it0;
+                for (int c = c_first; c < Rp; c += 32) {
+                    float sv[16], lv[16];
+                    tmem_ld16(s_addr + c, sv);
+                    if (!first_tile) tmem_ld16(tmem + lane_addr + col_l + c, lv);
+                    tmem_wait_ld();
+                    uint32_t w[8];
+#pragma unroll
+                    for (int e4 = 0; e4 < 4; ++e4) {
+                        const float4 mn = *reinterpret_cast<const float4 *>(&sh->mneg[c + 4 * e4]);
+                        float p0 = ex2_approx(fmaf(sv[4 * e4], sl2, mn.x)), p1 = ex2_approx(fmaf(sv[4 * e4 + 1], sl2, mn.y));
+                        float p2 = ex2_approx(fmaf(sv[4 * e4 + 2], sl2, mn.z)), p3 = ex2_approx(fmaf(sv[4 * e4 + 3], sl2, mn.w));
+                        if (tail) {   // uniform over the CTA
+                            const int4 lm = *reinterpret_cast<const int4 *>(&sh->limit[c + 4 * e4]);
+                            p0 = key <= lm.x ? p0 : 0.f; p1 = key <= lm.y ? p1 : 0.f;
+                            p2 = key <= lm.z ? p2 : 0.f; p3 = key <= lm.w ? p3 : 0.f;
+                        }
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1), h1 = __floats2bfloat162_rn(p2, p3);
+                        w[2 * e4] = *reinterpret_cast<uint32_t *>(&h0);
+                        w[2 * e4 + 1] = *reinterpret_cast<uint32_t *>(&h1);
+                        if (first_tile) { lv[4 * e4] = p0; lv[4 * e4 + 1] = p1; lv[4 * e4 + 2] = p2; lv[4 * e4 + 3] = p3; }
+                        else { lv[4 * e4] += p0; lv[4 * e4 + 1] += p1; lv[4 * e4 + 2] += p2; lv[4 * e4 + 3] += p3; }
+                    }
+                    tmem_st16(tmem + lane_addr + col_l + c, lv);
+                    *reinterpret_cast<uint4 *>(pk + (c >> 3) * (kBlockN * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(pk + ((c >> 3) + 1) * (kBlockN * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+                tmem_wait_st();
                 tc_fence_before();
+                mbar_arrive(smem_u32(&sh->s_free[j]));   // S^T buffer may be overwritten by QK of tile it+2
+                fence_proxy_async();
                 mbar_arrive(smem_u32(&sh->p_full[j]));
             }
-            if (!ok) break;
-            // ---- epilogue of the segment
-            if (n > 0) {
-                ok = W.wait(&sh->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1, 13);
-                if (!ok) break;
-                tc_fence_after();
+            if (aborted) break;
+            // ---- epilogue of the segment: row sums over the keys, then O^T / l
+            for (int c = c_first; c < Rp; c += 32) {
+                float lv[16];
+                tmem_ld16(tmem + lane_addr + col_l + c, lv);
+                tmem_wait_ld();
+                float mine = 0.f;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    float y = lv[e];
+#pragma unroll
+                    for (int o = 16; o; o >>= 1) y += __shfl_xor_sync(0xffffffffu, y, o);
+                    mine = (lane == e) ? y : mine;
+                }
+                if (lane < 16) sh->wpart[quarter][c + lane] = mine;
             }
-            if (warp_active) {
+            softmax_bar_sync();
+            if (st < Rp) sh->fscale[st] = (sh->wpart[0][st] + sh->wpart[1][st]) + (sh->wpart[2][st] + sh->wpart[3][st]);
+            ok = W.wait(&sh->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1, 13) && ok;
+            tc_fence_after();
+            softmax_bar_sync();
+            {
                 const int unit = b * Hkv + hk;
                 float *slot = p.partials + (size_t)(unit + blockIdx.x) * slot_float_count(R, D);
-                const int Rp = slot_rows_padded(R);
-                const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-                __nv_bfloat16 *og = (__nv_bfloat16 *)p.out + (((size_t)b * p.q_len + t_row) * p.n_q_heads + hk * G + g_row) * D;
-                float ov[32];
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    tmem_ld32(tmem + lane_addr + C::kColO + c * 32, ov);
+                const int Rpad = slot_rows_padded(R);
+                __nv_bfloat16 *og = (__nv_bfloat16 *)p.out;
+                for (int c = c_first; c < Rp; c += 32) {
+                    float ov[16];
+                    tmem_ld16(tmem + lane_addr + col_o + c, ov);
                     tmem_wait_ld();
-                    if (row_active) {
-                        if (whole_unit) {
+                    if (d_active && ok) {
 #pragma unroll
-                            for (int e = 0; e < 32; e += 8) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int x = 0; x < 4; ++x) {
-                                    __nv_bfloat162 h2 = __floats2bfloat162_rn(ov[e + 2 * x] * inv, ov[e + 2 * x + 1] * inv);
-                                    w[x] = *reinterpret_cast<uint32_t *>(&h2);
+                        for (int e = 0; e < 16; ++e) {
+                            const int r = c + e;
+                            if (r < R) {
+                                const float l = sh->fscale[r];
+                                const float m_ref = -sh->mneg[r];   // -inf while nothing was visible
+                                if (whole_unit) {
+                                    og[(size_t)sh->rowoff[r] * D + d] = __float2bfloat16_rn(l > 0.f ? ov[e] / l : 0.f);
+                                    if (p.lse && d == (r & (D - 1))) p.lse[sh->rowoff[r]] = l > 0.f ? m_ref * kLn2 + logf(l) : -INFINITY;
+                                } else {
+                                    slot[2 * Rpad + (size_t)r * D + d] = (m_ref == -INFINITY) ? 0.f : ov[e];
+                                    if (d == (r & (D - 1))) {
+                                        slot[r] = (m_ref == -INFINITY) ? -INFINITY : m_ref * kLn2;   // natural-log domain for the combine
+                                        slot[Rpad + r] = (m_ref == -INFINITY) ? 0.f : l;
+                                    }
                                 }
-                                *reinterpret_cast<uint4 *>(og + c * 32 + e) = make_uint4(w[0], w[1], w[2], w[3]);
                             }
-                        } else {
-                            float4 *dst = reinterpret_cast<float4 *>(slot + 2 * Rp + (size_t)r * D + c * 32);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) dst[e] = make_float4(ov[4 * e], ov[4 * e + 1], ov[4 * e + 2], ov[4 * e + 3]);
                         }
-                    }
-                }
-                if (row_active) {
-                    if (whole_unit) {
-                        if (p.lse) p.lse[((size_t)b * p.q_len + t_row) * p.n_q_heads + hk * G + g_row] =
-                            l_sum > 0.f ? m_ref * kLn2 + logf(l_sum) : -INFINITY;
-                    } else {
-                        slot[r] = (m_ref == -INFINITY) ? -INFINITY : m_ref * kLn2;   // natural-log domain for the combine
-                        slot[Rp + r] = l_sum;
                     }
                 }
             }
             tc_fence_before();
+            softmax_bar_sync();   // tables and tensor memory are rewritten by the next segment
             t += n;
             ++seg;
         }
@@ -497,7 +644,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -582,7 +729,7 @@ static int32_t make_map(CUtensorMap *m, const void *pool, long long rows, int D)
     if (!enc) return fail(HIPPO_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
     cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kBlockN};
+    cuuint32_t box[2] = {64, (cuuint32_t)kPageSize};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -593,7 +740,7 @@ static int32_t make_map(CUtensorMap *m, const void *pool, long long rows, int D)
 
 bool attn_tc_supported(const AttnParams &p, int dtype) {
     return dtype == HIPPO_DTYPE_BF16 && (p.head_dim == 64 || p.head_dim == 128) && p.batch <= kTcMaxBatch &&
-           p.rows <= kBlockM;
+           p.rows <= kMaxRows;
 }
 
 template <int D>
@@ -604,12 +751,17 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     if (rc != HIPPO_OK) return rc;
     rc = make_map(&vm, p.v_pages, rows, D);
     if (rc != HIPPO_OK) return rc;
+    const int Rp = (p.rows + 15) & ~15;
+    const TcSmemPlan plan = tc_smem_plan(D, Rp);
+    if (plan.slots < 3) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "attention: shared memory too small for %d packed rows", p.rows);
+    int tmem_cols = 32;
+    while (tmem_cols < 4 * Rp) tmem_cols *= 2;
     static bool attr_set = false;
     if (!attr_set) {
-        HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem_bytes<D>()));
+        HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
-    attn_tc_kernel<D><<<grid, kTcThreads, tc_smem_bytes<D>(), stream>>>(p, km, vm);
+    attn_tc_kernel<D><<<grid, kTcThreads, plan.total, stream>>>(p, km, vm, Rp, plan.slots, tmem_cols);
     count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     const int total_rows = p.batch * p.q_len * p.n_q_heads;

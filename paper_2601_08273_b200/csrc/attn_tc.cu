@@ -15,10 +15,13 @@
 // If not (the common case after the first tile) the stale reference is kept; otherwise the exact row maxima are
 // recomputed and O^T and the partial sums are rescaled in tensor memory.
 //
-// Work split.  The tiles of all (sequence, kv head) units form one flat list that is cut into gridDim.x equal
-// contiguous ranges (persistent CTAs, one per SM).  A CTA walks its range unit by unit ("segments"); for each
-// segment it produces either the final output (it owns the whole unit) or a partial (m, l, O) in slot unit+cta of
-// the workspace, which the combine kernel merges.
+// Work split (persistent CTAs, one per SM).  With no more (sequence, kv head) units than CTAs, every unit gets a
+// whole number of CTAs in proportion to its tile count (at least one; largest-remainder rounding) and each CTA
+// streams one contiguous range of its unit's tiles: one "segment" per CTA, no pipeline drain in the middle.  With
+// more units than CTAs the tiles of all units form one flat list cut into gridDim.x equal ranges, and a CTA walks
+// its range segment by segment.  A segment yields either the final output (it covers the whole unit) or a partial
+// (m, l, O) in a workspace slot; CTA 0 records per unit the first slot and the number of contributors, and the
+// combine kernel merges them.
 //
 // CTA = 10 warps: warp 0 TMA producer: ring of 2-page slots, alternately K and V of a tile, full/empty mbarriers;
 //                        a K slot is released as soon as QK^T has read it
@@ -40,6 +43,7 @@ constexpr int kBlockN = 128;           // keys per tile = two KV pages
 constexpr int kMaxRows = 128;          // packed rows (padded)
 constexpr int kMaxSlots = 12;
 constexpr int kTcMaxBatch = 256;       // per-sequence tile prefix lives in shared memory
+constexpr int kMaxAlignedUnits = 256;  // unit-aligned split: per-unit tables live in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;              // lazy rescale: only when a score exceeds the reference by > 2^8
@@ -149,6 +153,11 @@ struct TcShared {
     int limit[kMaxRows];        // last visible key of each packed row
     int rowoff[kMaxRows];       // (b*q_len + t)*H_q + h of each packed row, -1 for padding rows
     int tile_prefix[kTcMaxBatch + 1];  // only [0, batch] used
+    // unit-aligned split
+    int sum_base;
+    uint32_t rem[kMaxAlignedUnits];
+    int n_cta[kMaxAlignedUnits];
+    int cta_base[kMaxAlignedUnits + 1];
 };
 
 struct Waiter {
@@ -228,6 +237,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         mbar_init(smem_u32(&sh->q_free), 1);
         mbar_init(smem_u32(&sh->drain), 1);
         sh->abort = 0;
+        sh->sum_base = 0;
         int acc = 0;
         for (int b = 0; b < B; ++b) { sh->tile_prefix[b] = acc; acc += seq_tiles(p.kv_len[b], p.q_len); }
         sh->tile_prefix[B] = acc;
@@ -250,8 +260,75 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     Partition part;
     part.total = (long long)sh->tile_prefix[B] * Hkv;
     part.grid = gridDim.x;
-    const long long t_begin = part.total > 0 ? part.start_of(blockIdx.x) : 0;
-    const long long t_end = part.total > 0 ? part.start_of(blockIdx.x + 1) : 0;
+    const int U = B * Hkv;
+    const bool aligned = U <= (int)gridDim.x && U <= kMaxAlignedUnits;
+    long long t_begin = 0, t_end = 0;
+    int2 *unit_info = reinterpret_cast<int2 *>(p.counters);   // per unit: first slot, number of contributing CTAs
+    if (aligned) {
+        // CTAs per unit: one each, the others in proportion to the tile counts (largest remainders first)
+        const int my_tiles = tid < U ? sh->tile_prefix[tid / Hkv + 1] - sh->tile_prefix[tid / Hkv] : 0;
+        const bool live = my_tiles > 0;
+        const int n_live = __syncthreads_count(live);
+        const int spare = (int)gridDim.x - n_live;
+        int my_base = 0;
+        if (tid < U) {
+            uint32_t r = 0;
+            if (live) {
+                const long long num = (long long)spare * my_tiles;
+                my_base = (int)(num / part.total);
+                r = (uint32_t)(num % part.total);
+                if (my_base) atomicAdd(&sh->sum_base, my_base);
+            }
+            sh->rem[tid] = r;
+            sh->n_cta[tid] = live ? 1 : 0;
+        }
+        __syncthreads();
+        if (tid < U && live) {
+            const int leftover = spare - sh->sum_base;
+            const uint32_t r = sh->rem[tid];
+            int rank = 0;
+            for (int v = 0; v < U; ++v) rank += (sh->n_cta[v] && (sh->rem[v] > r || (sh->rem[v] == r && v < tid))) ? 1 : 0;
+            sh->n_cta[tid] = min(my_tiles, 1 + my_base + (rank < leftover ? 1 : 0));
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int acc = 0;
+            for (int u = 0; u < U; ++u) { sh->cta_base[u] = acc; acc += sh->n_cta[u]; }
+            sh->cta_base[U] = acc;
+        }
+        __syncthreads();
+        if (blockIdx.x == 0 && tid < U) unit_info[tid] = make_int2(sh->cta_base[tid], sh->n_cta[tid]);
+        if ((int)blockIdx.x < sh->cta_base[U]) {
+            int lo = 0, hi = U;   // largest u with cta_base[u] <= blockIdx.x
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (sh->cta_base[mid] <= (int)blockIdx.x) lo = mid; else hi = mid;
+            }
+            while (sh->n_cta[lo] == 0) ++lo;   // units without tiles share their neighbour's base
+            const int b = lo / Hkv, hk = lo % Hkv;
+            const long long T = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
+            const long long unit_start = (long long)sh->tile_prefix[b] * Hkv + hk * T;
+            const int i = (int)blockIdx.x - sh->cta_base[lo], nc = sh->n_cta[lo];
+            t_begin = unit_start + T * i / nc;
+            t_end = unit_start + T * (i + 1) / nc;
+        }
+    } else {
+        if (part.total > 0) { t_begin = part.start_of(blockIdx.x); t_end = part.start_of(blockIdx.x + 1); }
+        if (blockIdx.x == 0) {
+            for (int u = tid; u < U; u += kTcThreads) {
+                const int b = u / Hkv, hk = u % Hkv;
+                const long long T = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
+                int2 info = make_int2(0, 0);
+                if (T > 0) {
+                    const long long u0 = (long long)sh->tile_prefix[b] * Hkv + hk * T;
+                    const int c0 = part.cta_of(u0), c1 = part.cta_of(u0 + T - 1);
+                    info = make_int2(u + c0, c1 - c0 + 1);     // slot index = unit + cta
+                }
+                unit_info[u] = info;
+            }
+        }
+    }
+    const int slot_bias = aligned ? 0 : 1;   // slot = blockIdx.x (+ unit in the flat split)
 
     // Every role walks the same list of segments.  A segment = (b, hk, first tile, tile count) taken from the flat
     // range [t_begin, t_end); order is unit-major: all tiles of (b, hk=0), then (b, hk=1), ...
@@ -603,7 +680,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             softmax_bar_sync();
             {
                 const int unit = b * Hkv + hk;
-                float *slot = p.partials + (size_t)(unit + blockIdx.x) * slot_float_count(R, D);
+                float *slot = p.partials + (size_t)(slot_bias * unit + blockIdx.x) * slot_float_count(R, D);
                 const int Rpad = slot_rows_padded(R);
                 __nv_bfloat16 *og = (__nv_bfloat16 *)p.out;
                 for (int c = c_first; c < Rp; c += 32) {
@@ -653,7 +730,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
 // weights with lane-parallel loads, then thread d accumulates column d over the contributors with independent,
 // coalesced loads.
 template <int D>
-__global__ void __launch_bounds__(D) attn_tc_combine_kernel(const AttnParams p, int grid_main) {
+__global__ void __launch_bounds__(D) attn_tc_combine_kernel(const AttnParams p) {
     __shared__ float w_s[kExtraSlots];
     __shared__ float s_lse;
     const int R = p.rows, G = p.group, Hkv = p.n_kv_heads;
@@ -661,28 +738,17 @@ __global__ void __launch_bounds__(D) attn_tc_combine_kernel(const AttnParams p, 
     const int h = row % p.n_q_heads, t = (row / p.n_q_heads) % p.q_len, b = row / (p.n_q_heads * p.q_len);
     const int hk = h / G, r = t * G + (h % G);
     __nv_bfloat16 *out = (__nv_bfloat16 *)p.out + (size_t)row * D;
-    long long before = 0, total = 0;
-    for (int i = 0; i < p.batch; ++i) {
-        const int nt_i = seq_tiles(p.kv_len[i], p.q_len);
-        if (i < b) before += nt_i;
-        total += nt_i;
-    }
-    const int nt = seq_tiles(p.kv_len[b], p.q_len);
-    if (nt == 0) {
+    if (seq_tiles(p.kv_len[b], p.q_len) == 0) {
         out[tid] = __float2bfloat16_rn(0.f);
         if (p.lse && tid == 0) p.lse[row] = -INFINITY;
         return;
     }
-    Partition part;
-    part.total = total * Hkv;
-    part.grid = grid_main;
-    const long long u0 = before * Hkv + (long long)hk * nt, u1 = u0 + nt;
-    const int c0 = part.cta_of(u0), c1 = part.cta_of(u1 - 1);
-    if (c0 == c1) return;
-    const int n = c1 - c0 + 1;
+    const int2 info = reinterpret_cast<const int2 *>(p.counters)[b * Hkv + hk];   // first slot, contributors
+    const int n = info.y;
+    if (n <= 1) return;
     const size_t slot_floats = slot_float_count(R, D);
     const int Rp = slot_rows_padded(R);
-    const float *base = p.partials + (size_t)(b * Hkv + hk + c0) * slot_floats;   // slot index = unit + cta
+    const float *base = p.partials + (size_t)info.x * slot_floats;
     if (tid < 32) {
         float M = -INFINITY;
         for (int c = tid; c < n; c += 32) M = fmaxf(M, base[(size_t)c * slot_floats + r]);
@@ -765,7 +831,7 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     const int total_rows = p.batch * p.q_len * p.n_q_heads;
-    attn_tc_combine_kernel<D><<<total_rows, D, 0, stream>>>(p, grid);
+    attn_tc_combine_kernel<D><<<total_rows, D, 0, stream>>>(p);
     count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;

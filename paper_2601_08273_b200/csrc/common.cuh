@@ -46,7 +46,7 @@ __host__ __device__ inline size_t slot_float_count(int rows, int head_dim) {
     return 2 * (size_t)slot_rows_padded(rows) + (size_t)rows * head_dim;
 }
 
-// Layout of an attention workspace: header | arrival counters | partial slots.
+// Layout of an attention workspace: header | per-unit slot table | partial slots.
 struct AttnWsLayout {
     size_t counters_off, counters_bytes, partials_off, slot_floats, n_slots, total;
 };
@@ -54,7 +54,7 @@ inline AttnWsLayout attn_ws_layout(int batch, int q_len, int n_q_heads, int n_kv
     AttnWsLayout L;
     int rows = q_len * (n_q_heads / n_kv_heads);
     L.counters_off = kWsHeaderBytes;
-    L.counters_bytes = align_up((size_t)batch * n_kv_heads * sizeof(int32_t), 256);
+    L.counters_bytes = align_up((size_t)batch * n_kv_heads * 2 * sizeof(int32_t), 256);   // per unit: first slot, contributors
     L.partials_off = L.counters_off + L.counters_bytes;
     L.slot_floats = slot_float_count(rows, head_dim);
     L.n_slots = (size_t)batch * n_kv_heads + kExtraSlots;

@@ -82,6 +82,24 @@ def test_packed_row_shapes_bf16(hb, rows):
     check_full(hb, hb.hippo_verify_attention, q, k, v, lens, "bf16")
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_more_units_than_sms(hb, D):
+    """200 (sequence, kv head) units: more than one per SM, so CTAs walk several units and units straddle CTAs."""
+    rng = np.random.default_rng(23)
+    B, q_len, Hq, Hkv = 50, 3, 8, 4
+    lens = [int(x) for x in rng.integers(q_len, 900, size=B)]
+    lens[7], lens[8] = 1, 2                       # shorter than q_len: skipped, zero output
+    q = W.round_to_storage(rng.standard_normal((B, q_len, Hq, D)).astype(np.float32), "bf16")
+    k = W.round_to_storage(rng.standard_normal((B, max(lens), Hkv, D)).astype(np.float32), "bf16")
+    v = W.round_to_storage(rng.standard_normal((B, max(lens), Hkv, D)).astype(np.float32), "bf16")
+    got, lse = run_case(hb, hb.hippo_verify_attention, q, k, v, lens, "bf16", shuffle_seed=9)
+    live = [b for b in range(B) if lens[b] >= q_len]
+    ref, ref_lse = oracle.attention(q[live], k[live], v[live], [lens[b] for b in live])
+    assert_close(got[live], ref, TOL["bf16"], "many units")
+    assert_close(lse[live], ref_lse, 2e-3, "many units lse")
+    assert np.all(got[7:9] == 0) and np.all(np.isneginf(lse[7:9]))
+
+
 def test_short_sequence_is_skipped_and_zeroed(hb):
     rng = np.random.default_rng(3)
     B, q_len, Hq, Hkv, D = 2, 4, 4, 2, 64

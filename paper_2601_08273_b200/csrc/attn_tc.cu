@@ -223,6 +223,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = p.rows, G = p.group, Hkv = p.n_kv_heads, B = p.batch;
     const Waiter W{sh, p.header};
+    // Launched with programmatic stream serialization: the CTAs may be scheduled while the previous kernel of the
+    // stream drains; nothing is read or written before that kernel has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- set-up: barriers, tile prefix, tensor memory
     if (tid == 0) {
@@ -329,6 +332,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         }
     }
     const int slot_bias = aligned ? 0 : 1;   // slot = blockIdx.x (+ unit in the flat split)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel's CTAs may be scheduled
 
     // Every role walks the same list of segments.  A segment = (b, hk, first tile, tile count) taken from the flat
     // range [t_begin, t_end); order is unit-major: all tiles of (b, hk=0), then (b, hk=1), ...
@@ -725,21 +729,25 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     }
 }
 
-// Merge of the per-CTA partials of one output row (b, t, h); rows whose unit was owned by a single CTA were written
-// by it and are skipped.  One CTA of D threads per row: warp 0 turns the contributors' (m, l) into normalised
-// weights with lane-parallel loads, then thread d accumulates column d over the contributors with independent,
-// coalesced loads.
+// Merge of the per-CTA partials of one output row (b, t, h); rows whose unit was covered by a single CTA were
+// written by it and are skipped.  One CTA of 8 warps per row.  Warp w takes the contributors c = w, w+8, ... and
+// merges them online (running max, sum, D/32 output columns per lane); every global load of a pass is independent
+// of the others, so a pass costs one memory round trip.  The eight warp results are merged through shared memory.
+constexpr int kCombineThreads = 256;
 template <int D>
-__global__ void __launch_bounds__(D) attn_tc_combine_kernel(const AttnParams p) {
-    __shared__ float w_s[kExtraSlots];
-    __shared__ float s_lse;
+__global__ void __launch_bounds__(kCombineThreads) attn_tc_combine_kernel(const AttnParams p) {
+    constexpr int V = D / 32;   // output columns per lane
+    __shared__ float w_m[8], w_l[8];
+    __shared__ float w_acc[8][D];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int R = p.rows, G = p.group, Hkv = p.n_kv_heads;
-    const int row = blockIdx.x, tid = threadIdx.x;
+    const int row = blockIdx.x, tid = threadIdx.x, w = tid >> 5, lane = tid & 31;
     const int h = row % p.n_q_heads, t = (row / p.n_q_heads) % p.q_len, b = row / (p.n_q_heads * p.q_len);
     const int hk = h / G, r = t * G + (h % G);
     __nv_bfloat16 *out = (__nv_bfloat16 *)p.out + (size_t)row * D;
     if (seq_tiles(p.kv_len[b], p.q_len) == 0) {
-        out[tid] = __float2bfloat16_rn(0.f);
+        if (tid < D) out[tid] = __float2bfloat16_rn(0.f);
         if (p.lse && tid == 0) p.lse[row] = -INFINITY;
         return;
     }
@@ -749,29 +757,54 @@ __global__ void __launch_bounds__(D) attn_tc_combine_kernel(const AttnParams p) 
     const size_t slot_floats = slot_float_count(R, D);
     const int Rp = slot_rows_padded(R);
     const float *base = p.partials + (size_t)info.x * slot_floats;
-    if (tid < 32) {
-        float M = -INFINITY;
-        for (int c = tid; c < n; c += 32) M = fmaxf(M, base[(size_t)c * slot_floats + r]);
-        for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-        float L = 0.f;
-        for (int c = tid; c < n; c += 32) {
-            const float m = base[(size_t)c * slot_floats + r];
-            const float w = (m == -INFINITY) ? 0.f : expf(m - M);
-            w_s[c] = w;
-            L += base[(size_t)c * slot_floats + Rp + r] * w;
+    float M = -INFINITY, L = 0.f, acc[V];
+#pragma unroll
+    for (int x = 0; x < V; ++x) acc[x] = 0.f;
+    for (int c0 = w; c0 < n; c0 += 32) {
+        float m[4], l[4], v[4][V];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = min(c0 + 8 * j, n - 1);    // clamped; a repeated contributor is dropped below
+            const float *sl = base + (size_t)c * slot_floats;
+            m[j] = sl[r];
+            l[j] = sl[Rp + r];
+            if (V == 4) {
+                const float4 t4 = *reinterpret_cast<const float4 *>(sl + 2 * Rp + (size_t)r * D + lane * V);
+                v[j][0] = t4.x; v[j][1] = t4.y; v[j][V - 2] = t4.z; v[j][V - 1] = t4.w;
+            } else {
+                const float2 t2 = *reinterpret_cast<const float2 *>(sl + 2 * Rp + (size_t)r * D + lane * V);
+                v[j][0] = t2.x; v[j][1] = t2.y;
+            }
         }
-        for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        for (int c = tid; c < n; c += 32) w_s[c] *= inv;
-        if (tid == 0) s_lse = L > 0.f ? M + logf(L) : -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (c0 + 8 * j >= n || m[j] == -INFINITY) continue;
+            const float m_new = fmaxf(M, m[j]);
+            const float f_old = (M == -INFINITY) ? 0.f : expf(M - m_new), f_new = expf(m[j] - m_new);
+            L = L * f_old + l[j] * f_new;
+#pragma unroll
+            for (int x = 0; x < V; ++x) acc[x] = acc[x] * f_old + v[j][x] * f_new;
+            M = m_new;
+        }
     }
+    if (lane == 0) { w_m[w] = M; w_l[w] = L; }
+#pragma unroll
+    for (int x = 0; x < V; ++x) w_acc[w][lane * V + x] = acc[x];
     __syncthreads();
-    const float *o = base + 2 * Rp + (size_t)r * D + tid;
-    float acc = 0.f;
-#pragma unroll 8
-    for (int c = 0; c < n; ++c) acc = fmaf(o[(size_t)c * slot_floats], w_s[c], acc);
-    out[tid] = __float2bfloat16_rn(acc);
-    if (p.lse && tid == 0) p.lse[row] = s_lse;
+    if (tid < D) {
+        float Mt = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) Mt = fmaxf(Mt, w_m[k]);
+        float Lt = 0.f, o = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float f = (w_m[k] == -INFINITY) ? 0.f : expf(w_m[k] - Mt);
+            Lt += w_l[k] * f;
+            o += w_acc[k][tid] * f;
+        }
+        out[tid] = __float2bfloat16_rn(Lt > 0.f ? o / Lt : 0.f);
+        if (p.lse && tid == 0) p.lse[row] = Lt > 0.f ? Mt + logf(Lt) : -INFINITY;
+    }
 }
 
 // ---- host side -----------------------------------------------------------------------------------------------------
@@ -827,13 +860,25 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
         HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
-    attn_tc_kernel<D><<<grid, kTcThreads, plan.total, stream>>>(p, km, vm, Rp, plan.slots, tmem_cols);
+    // Both kernels are launched with programmatic stream serialization and wait (griddepcontrol.wait) before they
+    // touch memory, so stream order is kept while launch latency overlaps the previous kernel's tail.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = (size_t)plan.total;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols));
     count_launches(1);
-    HIPPO_CUDA_TRY(cudaGetLastError());
-    const int total_rows = p.batch * p.q_len * p.n_q_heads;
-    attn_tc_combine_kernel<D><<<total_rows, D, 0, stream>>>(p);
+    cfg.gridDim = dim3((unsigned)(p.batch * p.q_len * p.n_q_heads));
+    cfg.blockDim = dim3(kCombineThreads);
+    cfg.dynamicSmemBytes = 0;
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_combine_kernel<D>, p));
     count_launches(1);
-    HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;
 }
 

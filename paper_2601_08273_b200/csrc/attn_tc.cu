@@ -15,11 +15,17 @@
 // If not (the common case after the first tile) the stale reference is kept; otherwise the exact row maxima are
 // recomputed and O^T and the partial sums are rescaled in tensor memory.
 //
-// Work split (persistent CTAs, one per SM).  With no more (sequence, kv head) units than CTAs, every unit gets a
-// whole number of CTAs in proportion to its tile count (at least one; largest-remainder rounding) and each CTA
-// streams one contiguous range of its unit's tiles: one "segment" per CTA, no pipeline drain in the middle.  With
-// more units than CTAs the tiles of all units form one flat list cut into gridDim.x equal ranges, and a CTA walks
-// its range segment by segment.  A segment yields either the final output (it covers the whole unit) or a partial
+// Work split (persistent CTAs, one per SM).  Three modes, chosen on the host from the shape:
+//  * cluster: one thread-block cluster (2, 4, 8 or 16 CTAs) per unit.  The CTAs of a cluster split the unit's
+//    tiles evenly, leave their partial (m, l, O) in their own shared memory, and after a cluster barrier every CTA
+//    merges a share of the rows by reading its peers' partials through distributed shared memory.  One launch, no
+//    trip through global memory; used whenever clusters of that size keep enough SMs busy.
+//  * unit-aligned split + combine kernel: with no more (sequence, kv head) units than CTAs, every unit gets a
+//    whole number of CTAs in proportion to its tile count (at least one; largest-remainder rounding) and each CTA
+//    streams one contiguous range of its unit's tiles: one "segment" per CTA, no pipeline drain in the middle.
+//  * flat split + combine kernel: with more units than CTAs the tiles of all units form one flat list cut into
+//    gridDim.x equal ranges, and a CTA walks its range segment by segment.
+// Without clusters a segment yields either the final output (it covers the whole unit) or a partial
 // (m, l, O) in a workspace slot; CTA 0 records per unit the first slot and the number of contributors, and the
 // combine kernel merges them.
 //
@@ -109,6 +115,30 @@ __device__ __forceinline__ float warp_max(float x) {
     float y;
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_map(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 ld_cluster_v2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -208,7 +238,7 @@ static TcSmemPlan tc_smem_plan(int D, int Rp) {
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
-               const int Rp, const int n_slots, const int tmem_cols) {
+               const int Rp, const int n_slots, const int tmem_cols, const int cluster_size) {
     constexpr int kChunks = D / 64;                     // 64-column (128-byte) swizzle chunks per row
     constexpr int kPageBytes = kPageSize * D * 2;       // K or V of one page and head
     constexpr int kSlotBytes = 2 * kPageBytes;          // K or V of one tile
@@ -264,10 +294,18 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     part.total = (long long)sh->tile_prefix[B] * Hkv;
     part.grid = gridDim.x;
     const int U = B * Hkv;
-    const bool aligned = U <= (int)gridDim.x && U <= kMaxAlignedUnits;
+    const bool clustered = cluster_size > 1;                  // one cluster per unit, merge through shared memory
+    const bool aligned = !clustered && U <= (int)gridDim.x && U <= kMaxAlignedUnits;
     long long t_begin = 0, t_end = 0;
     int2 *unit_info = reinterpret_cast<int2 *>(p.counters);   // per unit: first slot, number of contributing CTAs
-    if (aligned) {
+    if (clustered) {
+        const int u = blockIdx.x / cluster_size, i = blockIdx.x % cluster_size;
+        const int b = u / Hkv, hk = u % Hkv;
+        const long long T = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
+        const long long unit_start = (long long)sh->tile_prefix[b] * Hkv + hk * T;
+        t_begin = unit_start + T * i / cluster_size;
+        t_end = unit_start + T * (i + 1) / cluster_size;
+    } else if (aligned) {
         // CTAs per unit: one each, the others in proportion to the tile counts (largest remainders first)
         const int my_tiles = tid < U ? sh->tile_prefix[tid / Hkv + 1] - sh->tile_prefix[tid / Hkv] : 0;
         const bool live = my_tiles > 0;
@@ -684,7 +722,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             softmax_bar_sync();
             {
                 const int unit = b * Hkv + hk;
-                float *slot = p.partials + (size_t)(slot_bias * unit + blockIdx.x) * slot_float_count(R, D);
+                // partial: a workspace slot, or (clustered) this CTA's ring memory, idle once the last PV has completed
+                float *slot = clustered ? reinterpret_cast<float *>(ring)
+                                        : p.partials + (size_t)(slot_bias * unit + blockIdx.x) * slot_float_count(R, D);
                 const int Rpad = slot_rows_padded(R);
                 __nv_bfloat16 *og = (__nv_bfloat16 *)p.out;
                 for (int c = c_first; c < Rp; c += 32) {
@@ -698,7 +738,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                             if (r < R) {
                                 const float l = sh->fscale[r];
                                 const float m_ref = -sh->mneg[r];   // -inf while nothing was visible
-                                if (whole_unit) {
+                                if (whole_unit && !clustered) {
                                     og[(size_t)sh->rowoff[r] * D + d] = __float2bfloat16_rn(l > 0.f ? ov[e] / l : 0.f);
                                     if (p.lse && d == (r & (D - 1))) p.lse[sh->rowoff[r]] = l > 0.f ? m_ref * kLn2 + logf(l) : -INFINITY;
                                 } else {
@@ -723,6 +763,66 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     // ---- teardown
     tc_fence_before();
     __syncthreads();
+    if (clustered) {
+        // Every thread of every CTA of the cluster gets here, whatever happened before, so the barriers complete.
+        const int u = blockIdx.x / cluster_size, rank = blockIdx.x % cluster_size;
+        const int b = u / Hkv, hk = u % Hkv;
+        const int Rpad = slot_rows_padded(R);
+        float *mine = reinterpret_cast<float *>(ring);
+        if (t_begin == t_end) {   // no tiles for this CTA: an empty partial
+            for (int r = tid; r < R; r += kTcThreads) { mine[r] = -INFINITY; mine[Rpad + r] = 0.f; }
+        }
+        cluster_sync_all();
+        if (sh->tile_prefix[b + 1] != sh->tile_prefix[b]) {
+            // rows r = rank, rank + cluster_size, ... of the unit are merged here, one warp per row
+            constexpr int V = D / 32;
+            const uint32_t local = smem_u32(mine);
+            for (int r = rank + cluster_size * warp; r < R; r += cluster_size * (kTcThreads / 32)) {
+                float M = -INFINITY, L = 0.f, acc[V];
+#pragma unroll
+                for (int x = 0; x < V; ++x) acc[x] = 0.f;
+                for (int c0 = 0; c0 < cluster_size; c0 += 8) {
+                    float m[8], l[8], v[8][V];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t peer = cluster_map(local, (uint32_t)min(c0 + j, cluster_size - 1));
+                        m[j] = ld_cluster_f32(peer + 4 * r);
+                        l[j] = ld_cluster_f32(peer + 4 * (Rpad + r));
+                        const uint32_t oa = peer + 4 * (2 * Rpad + r * D + lane * V);
+                        if (V == 4) {
+                            const float4 t4 = ld_cluster_v4(oa);
+                            v[j][0] = t4.x; v[j][1] = t4.y; v[j][V - 2] = t4.z; v[j][V - 1] = t4.w;
+                        } else {
+                            const float2 t2 = ld_cluster_v2(oa);
+                            v[j][0] = t2.x; v[j][1] = t2.y;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (c0 + j >= cluster_size || m[j] == -INFINITY) continue;
+                        const float m_new = fmaxf(M, m[j]);
+                        const float f_old = (M == -INFINITY) ? 0.f : expf(M - m_new), f_new = expf(m[j] - m_new);
+                        L = L * f_old + l[j] * f_new;
+#pragma unroll
+                        for (int x = 0; x < V; ++x) acc[x] = acc[x] * f_old + v[j][x] * f_new;
+                        M = m_new;
+                    }
+                }
+                const size_t ro = (size_t)(b * p.q_len + r / G) * p.n_q_heads + hk * G + r % G;
+                const float inv = L > 0.f ? 1.f / L : 0.f;
+                __nv_bfloat16 *o = (__nv_bfloat16 *)p.out + ro * D + lane * V;
+                if (V == 4) {
+                    __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv), h1 = __floats2bfloat162_rn(acc[V - 2] * inv, acc[V - 1] * inv);
+                    *reinterpret_cast<uint2 *>(o) = make_uint2(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1));
+                } else {
+                    __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
+                    *reinterpret_cast<uint32_t *>(o) = *reinterpret_cast<uint32_t *>(&h0);
+                }
+                if (p.lse && lane == 0) p.lse[ro] = L > 0.f ? M + logf(L) : -INFINITY;
+            }
+        }
+        cluster_sync_all();   // nobody leaves while a peer may still read its shared memory
+    }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
@@ -842,6 +942,20 @@ bool attn_tc_supported(const AttnParams &p, int dtype) {
            p.rows <= kMaxRows;
 }
 
+// Cluster size for the one-cluster-per-unit mode, or 0 for the split modes.  `tiles` = upper bound of the tiles of a
+// unit; max_active[cs] = clusters of cs CTAs of this kernel that the device keeps resident at once.  The cluster mode
+// needs no second kernel (worth about five tile times), but all clusters must be resident together and a unit gets
+// at most 16 SMs, so long caches with few units stay on the split path.
+static int choose_cluster_size(int units, int tiles, const int *max_active) {
+    int best = 0, best_cost = ceil_div(units * tiles, kNumSMs) + 5;
+    for (int cs = 2; cs <= 16 && cs <= tiles; ++cs) {
+        if (units > max_active[cs]) continue;
+        const int cost = ceil_div(tiles, cs);
+        if (cost < best_cost || (cost == best_cost && best == 0)) { best = cs; best_cost = cost; }
+    }
+    return best;
+}
+
 template <int D>
 static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     CUtensorMap km, vm;
@@ -858,21 +972,56 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     static bool attr_set = false;
     if (!attr_set) {
         HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
         attr_set = true;
     }
+    const int units = p.batch * p.n_kv_heads;
+    // resident clusters per cluster size, asked once per ring size (the only launch parameter that moves it)
+    static int max_active[kMaxSlots + 1][17];
+    static bool have_active[kMaxSlots + 1] = {false};
+    if (!have_active[plan.slots]) {
+        for (int c = 2; c <= 16; ++c) {
+            cudaLaunchConfig_t q = {};
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = (unsigned)c; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+            q.gridDim = dim3((unsigned)(c * kNumSMs)); q.blockDim = dim3(kTcThreads); q.dynamicSmemBytes = (size_t)plan.total;
+            q.attrs = qa; q.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<D>, &q) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
+            max_active[plan.slots][c] = n;
+        }
+        have_active[plan.slots] = true;
+    }
+    const int cs = p.num_splits > 0 ? 0 : choose_cluster_size(units, ceil_div(p.max_kv_len, kBlockN), max_active[plan.slots]);
     // Both kernels are launched with programmatic stream serialization and wait (griddepcontrol.wait) before they
     // touch memory, so stream order is kept while launch latency overlaps the previous kernel's tail.
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kTcThreads);
     cfg.dynamicSmemBytes = (size_t)plan.total;
     cfg.stream = stream;
     cfg.attrs = attr;
+    if (cs > 1) {
+        // one cluster per unit; the partial of a CTA (m, l, O) must fit in its ring memory
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cs;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+        cfg.gridDim = dim3((unsigned)(units * cs));
+        if (slot_float_count(p.rows, D) * sizeof(float) <= (size_t)plan.slots * kBlockN * D * 2 &&
+            cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols, cs) == cudaSuccess) {
+            count_launches(1);
+            return HIPPO_OK;
+        }
+        (void)cudaGetLastError();   // clusters of this size cannot be scheduled here: use the split modes
+    }
     cfg.numAttrs = 1;
-    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols));
+    cfg.gridDim = dim3((unsigned)grid);
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols, 0));
     count_launches(1);
     cfg.gridDim = dim3((unsigned)(p.batch * p.q_len * p.n_q_heads));
     cfg.blockDim = dim3(kCombineThreads);

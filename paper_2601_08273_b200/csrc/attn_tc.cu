@@ -190,25 +190,31 @@ struct TcShared {
     int cta_base[kMaxAlignedUnits + 1];
 };
 
+// The polling part of a bounded wait, kept out of line: it is entered only when the barrier is not yet complete and
+// would otherwise be replicated at some twenty call sites.
+__device__ __noinline__ bool wait_slow(TcShared *sh, WsHeader *hdr, uint32_t b, uint32_t parity, int site) {
+    const unsigned long long t0 = global_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(b, parity)) return true;
+        if ((i & 31) == 0) {
+            if (sh->abort) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                sh->abort = 1;
+                atomicExch(&hdr->status, (int)HIPPO_ERR_TIMEOUT);
+                hdr->where = site;
+                return false;
+            }
+        }
+    }
+}
+
 struct Waiter {
     TcShared *sh;
     WsHeader *hdr;
     __device__ __forceinline__ bool wait(unsigned long long *bar, uint32_t parity, int site) const {
         const uint32_t b = smem_u32(bar);
         if (mbar_try_wait(b, parity)) return true;
-        const unsigned long long t0 = global_ns();
-        for (uint32_t i = 1;; ++i) {
-            if (mbar_try_wait(b, parity)) return true;
-            if ((i & 31) == 0) {
-                if (sh->abort) return false;
-                if (global_ns() - t0 > kWaitLimitNs) {
-                    sh->abort = 1;
-                    atomicExch(&hdr->status, (int)HIPPO_ERR_TIMEOUT);
-                    hdr->where = site;
-                    return false;
-                }
-            }
-        }
+        return wait_slow(sh, hdr, b, parity, site);
     }
 };
 
@@ -258,22 +264,20 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- set-up: barriers, tile prefix, tensor memory
-    if (tid == 0) {
-        for (int s = 0; s < n_slots; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
-        for (int j = 0; j < 2; ++j) {
-            mbar_init(smem_u32(&sh->s_full[j]), 1);
-            mbar_init(smem_u32(&sh->s_free[j]), kSoftmaxThreads);
-            mbar_init(smem_u32(&sh->p_full[j]), kSoftmaxThreads);
-            mbar_init(smem_u32(&sh->pv_done[j]), 1);
-        }
-        mbar_init(smem_u32(&sh->q_full), kSoftmaxThreads);
-        mbar_init(smem_u32(&sh->q_free), 1);
-        mbar_init(smem_u32(&sh->drain), 1);
-        sh->abort = 0;
-        sh->sum_base = 0;
-        int acc = 0;
-        for (int b = 0; b < B; ++b) { sh->tile_prefix[b] = acc; acc += seq_tiles(p.kv_len[b], p.q_len); }
-        sh->tile_prefix[B] = acc;
+    {
+        // one barrier per thread: [0, n_slots) full, [n_slots, 2 n_slots) empty, then the fixed ones
+        const int nb = 2 * n_slots;
+        if (tid < nb) mbar_init(smem_u32(tid < n_slots ? &sh->full[tid] : &sh->empty[tid - n_slots]), 1);
+        else if (tid < nb + 2) mbar_init(smem_u32(&sh->s_full[tid - nb]), 1);
+        else if (tid < nb + 4) mbar_init(smem_u32(&sh->s_free[tid - nb - 2]), kSoftmaxThreads);
+        else if (tid < nb + 6) mbar_init(smem_u32(&sh->p_full[tid - nb - 4]), kSoftmaxThreads);
+        else if (tid < nb + 8) mbar_init(smem_u32(&sh->pv_done[tid - nb - 6]), 1);
+        else if (tid == nb + 8) mbar_init(smem_u32(&sh->q_full), kSoftmaxThreads);
+        else if (tid == nb + 9) mbar_init(smem_u32(&sh->q_free), 1);
+        else if (tid == nb + 10) mbar_init(smem_u32(&sh->drain), 1);
+        else if (tid == nb + 11) { sh->abort = 0; sh->sum_base = 0; }
+        // tiles per sequence, then an exclusive prefix
+        for (int b = tid; b < B; b += kTcThreads) sh->tile_prefix[b + 1] = seq_tiles(p.kv_len[b], p.q_len);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid == 32) {
@@ -285,6 +289,12 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int b = 0; b < B; ++b) { const int n = sh->tile_prefix[b + 1]; sh->tile_prefix[b] = acc; acc += n; }
+        sh->tile_prefix[B] = acc;
+    }
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh->tmem_base;

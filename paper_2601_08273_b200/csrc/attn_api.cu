@@ -57,6 +57,7 @@ static int32_t attention_entry(const char *who, bool draft_policy, int32_t batch
     p.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kv->head_dim);
     cudaStream_t s = (cudaStream_t)stream;
 
+    if (attn_small_supported(p, kv->dtype)) return launch_attn_small(p, s);   // few rows, short cache: latency-bound
     if (attn_tc_supported(p, kv->dtype)) {
         p.num_splits = num_splits;
         return launch_attn_tc(p, draft_policy, s);

@@ -94,5 +94,7 @@ int32_t launch_attn_generic(const AttnParams &p, int dtype, cudaStream_t stream)
 int32_t launch_attn_combine(const AttnParams &p, int dtype, int n_splits, cudaStream_t stream);
 int32_t launch_attn_tc(const AttnParams &p, bool draft_policy, cudaStream_t stream);
 bool attn_tc_supported(const AttnParams &p, int dtype);
+int32_t launch_attn_small(const AttnParams &p, cudaStream_t stream);
+bool attn_small_supported(const AttnParams &p, int dtype);
 
 }  // namespace hippo

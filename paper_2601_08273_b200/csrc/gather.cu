@@ -4,9 +4,10 @@
 // draft keeps only the chosen visual tokens plus the always-kept positions.  A pure copy, bound by HBM bandwidth:
 // per kept token and layer 2 * n_kv_heads * head_dim elements are read and written once.
 //
-// One thread moves 16 bytes.  Work items are ordered (chunk within row, destination token, head, K|V, layer) so that
-// consecutive threads write consecutive addresses of one destination (page, head) block; reads are whole rows of
-// head_dim elements (128 B for head_dim 64 bf16) scattered over the source pages.
+// One work item moves 16 bytes; a thread takes four items per round, all four loads issued before the first store.
+// Items are ordered (chunk within row, destination token, head) inside a (layer, K|V) plane given by blockIdx.y, so
+// that consecutive threads write consecutive addresses of one destination (page, head) block; reads are whole rows of
+// head_dim elements (128 B for head_dim 64 bf16) scattered over the source pages.  Index arithmetic is 32-bit.
 #include "common.cuh"
 
 namespace hippo {
@@ -19,33 +20,46 @@ struct GatherParams {
     int n_layers, batch, total_keep, n_kv_heads, row_chunks, src_mpps, dst_mpps;
 };
 
-__global__ void __launch_bounds__(256) gather_kv_kernel(const GatherParams p) {
-    const long long per_layer_kv = (long long)p.total_keep * p.n_kv_heads * p.row_chunks;
-    const long long total = per_layer_kv * 2 * p.n_layers;
-    const size_t row_bytes = (size_t)p.row_chunks * 16;
-    for (long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x; w < total; w += (long long)gridDim.x * blockDim.x) {
-        long long x = w;
-        const int c = (int)(x % p.row_chunks); x /= p.row_chunks;
-        const int i = (int)(x % p.total_keep); x /= p.total_keep;
-        const int h = (int)(x % p.n_kv_heads); x /= p.n_kv_heads;
-        const int is_v = (int)(x & 1);
-        const int l = (int)(x >> 1);
-        // sequence of flat keep index i: largest b with keep_offsets[b] <= i
-        int lo = 0, hi = p.batch;
-        while (hi - lo > 1) {
-            int mid = (lo + hi) >> 1;
-            if (p.keep_offsets[mid] <= i) lo = mid; else hi = mid;
+constexpr int kGatherThreads = 256;
+constexpr int kGatherUnroll = 4;
+
+__global__ void __launch_bounds__(kGatherThreads) gather_kv_kernel(const GatherParams p) {
+    const uint32_t per_plane = (uint32_t)p.total_keep * (uint32_t)p.n_kv_heads * (uint32_t)p.row_chunks;
+    const int l = blockIdx.y >> 1, is_v = blockIdx.y & 1;
+    const char *src = (is_v ? p.src_v : p.src_k) + (size_t)l * p.src_layer_stride;
+    char *dst = (is_v ? p.dst_v : p.dst_k) + (size_t)l * p.dst_layer_stride;
+    const uint32_t row_bytes = (uint32_t)p.row_chunks * 16u;
+    const uint32_t stride = gridDim.x * kGatherThreads;
+    for (uint32_t w0 = blockIdx.x * kGatherThreads + threadIdx.x; w0 < per_plane; w0 += stride * kGatherUnroll) {
+        size_t so[kGatherUnroll], dof[kGatherUnroll];
+        bool live[kGatherUnroll];
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const uint32_t w = w0 + u * stride;
+            live[u] = w < per_plane;
+            const uint32_t x = live[u] ? w : 0u;
+            const uint32_t c = x % (uint32_t)p.row_chunks, y = x / (uint32_t)p.row_chunks;
+            const int i = (int)(y % (uint32_t)p.total_keep), h = (int)(y / (uint32_t)p.total_keep);
+            // sequence of flat keep index i: largest b with keep_offsets[b] <= i
+            int lo = 0, hi = p.batch;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (__ldg(p.keep_offsets + mid) <= i) lo = mid; else hi = mid;
+            }
+            const int src_tok = __ldg(p.keep_idx + i);
+            const int dst_tok = i - __ldg(p.keep_offsets + lo);
+            const int sp = page_of(p.src_table, p.src_mpps, lo, src_tok / kPageSize);
+            const int dp = page_of(p.dst_table, p.dst_mpps, lo, dst_tok / kPageSize);
+            so[u] = (((size_t)sp * p.n_kv_heads + h) * kPageSize + (src_tok % kPageSize)) * row_bytes + c * 16u;
+            dof[u] = (((size_t)dp * p.n_kv_heads + h) * kPageSize + (dst_tok % kPageSize)) * row_bytes + c * 16u;
         }
-        const int b = lo;
-        const int src_tok = p.keep_idx[i];
-        const int dst_tok = i - p.keep_offsets[b];
-        const int sp = page_of(p.src_table, p.src_mpps, b, src_tok / kPageSize);
-        const int dp = page_of(p.dst_table, p.dst_mpps, b, dst_tok / kPageSize);
-        const size_t so = (((size_t)sp * p.n_kv_heads + h) * kPageSize + (src_tok % kPageSize)) * row_bytes + (size_t)c * 16;
-        const size_t d_o = (((size_t)dp * p.n_kv_heads + h) * kPageSize + (dst_tok % kPageSize)) * row_bytes + (size_t)c * 16;
-        const char *s = (is_v ? p.src_v : p.src_k) + (size_t)l * p.src_layer_stride + so;
-        char *d = (is_v ? p.dst_v : p.dst_k) + (size_t)l * p.dst_layer_stride + d_o;
-        *reinterpret_cast<uint4 *>(d) = __ldg(reinterpret_cast<const uint4 *>(s));
+        uint4 v[kGatherUnroll];
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u)
+            if (live[u]) v[u] = __ldg(reinterpret_cast<const uint4 *>(src + so[u]));
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u)
+            if (live[u]) *reinterpret_cast<uint4 *>(dst + dof[u]) = v[u];
     }
 }
 
@@ -92,11 +106,15 @@ extern "C" int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src
     p.src_layer_stride = src_layer_stride_bytes; p.dst_layer_stride = dst_layer_stride_bytes;
     p.n_layers = n_layers; p.batch = batch; p.total_keep = total_keep; p.n_kv_heads = src->n_kv_heads;
     p.row_chunks = (int)(row_bytes / 16); p.src_mpps = src->max_pages_per_seq; p.dst_mpps = dst->max_pages_per_seq;
-    const long long total = (long long)total_keep * p.n_kv_heads * p.row_chunks * 2 * n_layers;
-    long long blocks = (total + 255) / 256;
-    const long long cap = (long long)kNumSMs * 32;
-    if (blocks > cap) blocks = cap;
-    gather_kv_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(p);
+    const long long per_plane = (long long)total_keep * p.n_kv_heads * p.row_chunks;
+    if (per_plane > 0x7fffffffLL) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_gather_kv: more than 2^31 16-byte items per layer");
+    if (2 * n_layers > 65535) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_gather_kv: too many layers for one launch");
+    // blocks per (layer, K|V) plane: enough rounds of kGatherUnroll items per thread, at most ~16 blocks per SM in total
+    long long bx = (per_plane + kGatherThreads * kGatherUnroll - 1) / (kGatherThreads * kGatherUnroll);
+    const long long cap = (long long)kNumSMs * 16 / (2 * n_layers) + 1;
+    if (bx > cap) bx = cap;
+    if (bx < 1) bx = 1;
+    gather_kv_kernel<<<dim3((unsigned)bx, (unsigned)(2 * n_layers)), kGatherThreads, 0, (cudaStream_t)stream>>>(p);
     count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;

@@ -210,7 +210,7 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
  *     time on the GPU (different streams without an ordering between them) race on it and corrupt each other's
  *     result.  Order them, or give one of them hippo_accept with its own workspace.
  */
-#define HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES (256u * 1024u)
+#define HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES (1024u * 1024u)
 int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vocab, const float *target_logits,
                              const float *draft_logits, const int32_t *draft_tokens, const float *u_accept,
                              const float *u_resample, int32_t mode, int32_t *n_accepted, int32_t *out_tokens,

@@ -74,7 +74,7 @@ lib.hippo_accept.restype = _i32
 lib.hippo_accept.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp]
 lib.hippo_accept_noalloc.restype = _i32
 lib.hippo_accept_noalloc.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
-ACCEPT_NOALLOC_SCRATCH_BYTES = 256 * 1024
+ACCEPT_NOALLOC_SCRATCH_BYTES = 1024 * 1024
 
 
 class HippoError(RuntimeError):

@@ -6,11 +6,14 @@
 //   draw = inverse CDF in ascending token id: smallest t with cumsum_t > u_resample * total
 //
 // All probabilities, normalisers and CDFs are fp64 so that the decisions agree with an fp64 reference unless a
-// uniform lands within ~1e-15 of a boundary.  Four small kernels over the vocabulary:
+// uniform lands within ~1e-15 of a boundary.  Three kernels over the vocabulary, chained with programmatic
+// dependent launches (each waits for its predecessor before it reads anything):
 //   stats   per (sequence, logit row, 4096-token chunk): max and sum of exponentials
-//   decide  per sequence: merge the chunk stats, run the accept tests, store n and the two normalisers of row n
-//   wsum    per (sequence, chunk): total residual (or bonus) weight of the chunk, by the same in-order scan as `pick`
-//   pick    per sequence: locate the chunk, then the token, where the CDF crosses u * total
+//   weigh   per (sequence, chunk): every CTA merges the chunk stats of its sequence and runs the accept tests
+//           itself (a few hundred values; cheaper than a launch of its own), then scans the residual (or bonus)
+//           weights of its chunk in token order and stores the running sum after each thread's 16 tokens
+//   pick    per sequence: locate the chunk, then the 16-token group, then the token where the CDF crosses
+//           u * total; only that one group's weights are evaluated again
 #include <math.h>
 
 #include <mutex>
@@ -22,9 +25,10 @@ namespace hippo {
 constexpr int kAccThreads = 256;
 constexpr int kAccPerThread = 16;
 constexpr int kAccChunk = kAccThreads * kAccPerThread;  // 4096 vocabulary entries per chunk
+constexpr int kAccMaxRows = 2 * 64 + 1;
 
 struct RowInfo {
-    double Mp, Zp, Mq, Zq;  // max logit and sum of exponentials of target row n / draft row n
+    double Mp, Zp, Mq, Zq;  // max logit and 1 / (sum of exponentials) of target row n / draft row n
     int32_t n;              // accepted count
     int32_t bonus;          // 1: n == gamma, draw from P_gamma
     int32_t pad[2];
@@ -36,6 +40,7 @@ struct AcceptParams {
     int32_t *n_acc, *out;
     double2 *stats;  // [B][2*gamma+1][n_chunks]: (max, sum exp)
     double *wsum;    // [B][n_chunks]
+    double *tscan;   // [B][n_chunks][kAccThreads]: in-chunk running sum after each thread's tokens
     RowInfo *info;   // [B]
     int B, gamma, V, n_chunks;
 };
@@ -44,6 +49,9 @@ __device__ __forceinline__ const float *logit_row(const AcceptParams &p, int b, 
     // r in [0, gamma]: target row r; r in (gamma, 2*gamma]: draft row r - gamma - 1
     return r <= p.gamma ? p.tl + ((size_t)b * (p.gamma + 1) + r) * p.V : p.dl + ((size_t)b * p.gamma + (r - p.gamma - 1)) * p.V;
 }
+
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // In-order inclusive scan over the block's threads (thread i holds element i).  Deterministic.
 __device__ double block_scan_inclusive(double v, double *warp_tot /* [8] shared */, double *total) {
@@ -67,16 +75,28 @@ __device__ double block_scan_inclusive(double v, double *warp_tot /* [8] shared 
 __global__ void __launch_bounds__(kAccThreads) accept_stats_kernel(const AcceptParams p) {
     __shared__ float smax[kAccThreads / 32];
     __shared__ double ssum[kAccThreads / 32];
+    pdl_wait();
+    pdl_trigger();
     const int c = blockIdx.x, r = blockIdx.y, b = blockIdx.z, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float *row = logit_row(p, b, r);
     float v[kAccPerThread];
     float m = -INFINITY;
+    if ((c + 1) * kAccChunk <= p.V && (((uintptr_t)row) & 15) == 0 && (p.V & 3) == 0) {
+        // full chunk, 16-byte aligned: four float4 loads per thread
 #pragma unroll
-    for (int e = 0; e < kAccPerThread; ++e) {
-        int t = c * kAccChunk + e * kAccThreads + tid;
-        v[e] = t < p.V ? row[t] : -INFINITY;
-        m = fmaxf(m, v[e]);
+        for (int e4 = 0; e4 < kAccPerThread / 4; ++e4) {
+            const float4 t = __ldg(reinterpret_cast<const float4 *>(row + c * kAccChunk) + e4 * kAccThreads + tid);
+            v[4 * e4] = t.x; v[4 * e4 + 1] = t.y; v[4 * e4 + 2] = t.z; v[4 * e4 + 3] = t.w;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < kAccPerThread; ++e) {
+            const int t = c * kAccChunk + e * kAccThreads + tid;
+            v[e] = t < p.V ? row[t] : -INFINITY;
+        }
     }
+#pragma unroll
+    for (int e = 0; e < kAccPerThread; ++e) m = fmaxf(m, v[e]);
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if (lane == 0) smax[warp] = m;
     __syncthreads();
@@ -96,9 +116,55 @@ __global__ void __launch_bounds__(kAccThreads) accept_stats_kernel(const AcceptP
     }
 }
 
-__global__ void __launch_bounds__(kAccThreads) accept_decide_kernel(const AcceptParams p) {
-    extern __shared__ double rowstat[];  // [2*gamma+1][2]: M, Z
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+// Weight of token t in the distribution the emitted token is drawn from.  use_target_only: bonus row, or the
+// degenerate rejection with P_n == Q_n everywhere.
+__device__ __forceinline__ double weight_of(float tl, float dl, const RowInfo &ri, bool use_target_only) {
+    const double P = exp((double)tl - ri.Mp) * ri.Zp;
+    if (use_target_only) return P;
+    const double Q = exp((double)dl - ri.Mq) * ri.Zq;
+    const double w = P - Q;
+    return w > 0.0 ? w : 0.0;
+}
+__device__ __forceinline__ double draw_weight(const float *trow, const float *drow, int t, const RowInfo &ri, bool use_target_only) {
+    return weight_of(trow[t], use_target_only ? 0.f : drow[t], ri, use_target_only);
+}
+
+// Thread-local weights of one chunk (16 consecutive tokens per thread) and their in-order sum.
+__device__ __forceinline__ double chunk_local(const float *trow, const float *drow, int c, int V, const RowInfo &ri,
+                                              bool target_only, double *w) {
+    double s = 0.0;
+    const int t0 = c * kAccChunk + threadIdx.x * kAccPerThread;
+    float tv[kAccPerThread], dv[kAccPerThread];
+    const bool vec = t0 + kAccPerThread <= V && (((uintptr_t)(trow + t0) | (target_only ? 0 : (uintptr_t)(drow + t0))) & 15) == 0;
+    if (vec) {
+#pragma unroll
+        for (int e4 = 0; e4 < kAccPerThread / 4; ++e4) {
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(trow + t0) + e4);
+            tv[4 * e4] = a.x; tv[4 * e4 + 1] = a.y; tv[4 * e4 + 2] = a.z; tv[4 * e4 + 3] = a.w;
+            float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (!target_only) d = __ldg(reinterpret_cast<const float4 *>(drow + t0) + e4);
+            dv[4 * e4] = d.x; dv[4 * e4 + 1] = d.y; dv[4 * e4 + 2] = d.z; dv[4 * e4 + 3] = d.w;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < kAccPerThread; ++e) {
+            const int t = t0 + e;
+            tv[e] = t < V ? trow[t] : 0.f;
+            dv[e] = (t < V && !target_only) ? drow[t] : 0.f;
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < kAccPerThread; ++e) {
+        w[e] = t0 + e < V ? weight_of(tv[e], dv[e], ri, target_only) : 0.0;
+        s += w[e];
+    }
+    return s;
+}
+
+// Merge of the chunk statistics of every logit row of sequence b and the sequential accept tests.  Run by all
+// threads of a block; the result is identical in every block of the sequence (same data, same order).
+__device__ RowInfo decide_rows(const AcceptParams &p, int b, double *rowstat /* shared [2*gamma+1][2] */, int *s_n) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_rows = 2 * p.gamma + 1;
     for (int r = warp; r < n_rows; r += kAccThreads / 32) {
         const double2 *st = p.stats + ((size_t)b * n_rows + r) * p.n_chunks;
@@ -112,83 +178,80 @@ __global__ void __launch_bounds__(kAccThreads) accept_decide_kernel(const Accept
         if (lane == 0) { rowstat[2 * r] = M; rowstat[2 * r + 1] = Z; }
     }
     __syncthreads();
-    if (tid == 0) {
+    if (warp == 0) {
+        // lane j tests draft token j (all loads independent), then the first failing lane is n
+        const int32_t *x = p.x + (size_t)b * p.gamma;
+        int n = p.gamma;
+        for (int j0 = 0; j0 < p.gamma; j0 += 32) {
+            const int j = j0 + lane;
+            bool accept = true;
+            if (j < p.gamma) {
+                const int rq = p.gamma + 1 + j, tok = x[j];
+                const double P = exp((double)logit_row(p, b, j)[tok] - rowstat[2 * j]) / rowstat[2 * j + 1];
+                const double Q = exp((double)logit_row(p, b, rq)[tok] - rowstat[2 * rq]) / rowstat[2 * rq + 1];
+                const double u = (double)p.ua[(size_t)b * p.gamma + j];
+                accept = u * Q < P;
+            }
+            const unsigned rejected = __ballot_sync(0xffffffffu, !accept);
+            if (rejected) { n = j0 + __ffs(rejected) - 1; break; }
+        }
+        if (lane == 0) *s_n = n;
+    }
+    __syncthreads();
+    RowInfo ri;
+    ri.n = *s_n;
+    ri.bonus = (ri.n == p.gamma);
+    ri.Mp = rowstat[2 * ri.n]; ri.Zp = 1.0 / rowstat[2 * ri.n + 1];
+    if (ri.n < p.gamma) { ri.Mq = rowstat[2 * (p.gamma + 1 + ri.n)]; ri.Zq = 1.0 / rowstat[2 * (p.gamma + 1 + ri.n) + 1]; }
+    else { ri.Mq = 0.0; ri.Zq = 1.0; }
+    ri.pad[0] = ri.pad[1] = 0;
+    return ri;
+}
+
+__global__ void __launch_bounds__(kAccThreads) accept_weigh_kernel(const AcceptParams p) {
+    __shared__ double rowstat[2 * kAccMaxRows];
+    __shared__ double warp_tot[kAccThreads / 32];
+    __shared__ int s_n;
+    pdl_wait();
+    pdl_trigger();
+    const int c = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const RowInfo ri = decide_rows(p, b, rowstat, &s_n);
+    if (c == 0 && tid == 0) {
         const int32_t *x = p.x + (size_t)b * p.gamma;
         int32_t *out = p.out + (size_t)b * (p.gamma + 1);
-        int n = 0;
-        for (; n < p.gamma; ++n) {
-            const int rq = p.gamma + 1 + n;
-            const double P = exp((double)logit_row(p, b, n)[x[n]] - rowstat[2 * n]) / rowstat[2 * n + 1];
-            const double Q = exp((double)logit_row(p, b, rq)[x[n]] - rowstat[2 * rq]) / rowstat[2 * rq + 1];
-            const double u = (double)p.ua[(size_t)b * p.gamma + n];
-            if (!(u * Q < P)) break;
-            out[n] = x[n];
-        }
-        for (int j = n; j <= p.gamma; ++j) out[j] = -1;  // out[n] is filled by the pick kernel
-        p.n_acc[b] = n;
-        RowInfo ri;
-        ri.n = n;
-        ri.bonus = (n == p.gamma);
-        ri.Mp = rowstat[2 * n]; ri.Zp = rowstat[2 * n + 1];
-        if (n < p.gamma) { ri.Mq = rowstat[2 * (p.gamma + 1 + n)]; ri.Zq = rowstat[2 * (p.gamma + 1 + n) + 1]; }
-        else { ri.Mq = 0.0; ri.Zq = 1.0; }
-        ri.pad[0] = ri.pad[1] = 0;
+        for (int j = 0; j < ri.n; ++j) out[j] = x[j];
+        for (int j = ri.n; j <= p.gamma; ++j) out[j] = -1;  // out[n] is filled by the pick kernel
+        p.n_acc[b] = ri.n;
         p.info[b] = ri;
     }
-}
-
-// Weight of token t in the distribution the emitted token is drawn from.  use_target_only: bonus row, or the
-// degenerate rejection with P_n == Q_n everywhere.
-__device__ __forceinline__ double draw_weight(const float *trow, const float *drow, int t, const RowInfo &ri, bool use_target_only) {
-    const double P = exp((double)trow[t] - ri.Mp) / ri.Zp;
-    if (use_target_only) return P;
-    const double Q = exp((double)drow[t] - ri.Mq) / ri.Zq;
-    const double w = P - Q;
-    return w > 0.0 ? w : 0.0;
-}
-
-// Thread-local weights of one chunk (16 consecutive tokens per thread) and their in-order sum.
-__device__ __forceinline__ double chunk_local(const float *trow, const float *drow, int c, int V, const RowInfo &ri,
-                                              bool target_only, double *w) {
-    double s = 0.0;
-    const int t0 = c * kAccChunk + threadIdx.x * kAccPerThread;
-#pragma unroll
-    for (int e = 0; e < kAccPerThread; ++e) {
-        const int t = t0 + e;
-        w[e] = t < V ? draw_weight(trow, drow, t, ri, target_only) : 0.0;
-        s += w[e];
-    }
-    return s;
-}
-
-__global__ void __launch_bounds__(kAccThreads) accept_wsum_kernel(const AcceptParams p) {
-    __shared__ double warp_tot[kAccThreads / 32];
-    const int c = blockIdx.x, b = blockIdx.y;
-    const RowInfo ri = p.info[b];
     const float *trow = logit_row(p, b, ri.n);
     const float *drow = ri.bonus ? nullptr : logit_row(p, b, p.gamma + 1 + ri.n);
     double w[kAccPerThread], total;
     double s = chunk_local(trow, drow, c, p.V, ri, ri.bonus != 0, w);
-    block_scan_inclusive(s, warp_tot, &total);
-    if (threadIdx.x == 0) p.wsum[(size_t)b * p.n_chunks + c] = total;
+    const double incl = block_scan_inclusive(s, warp_tot, &total);
+    p.tscan[((size_t)b * p.n_chunks + c) * kAccThreads + tid] = incl;
+    if (tid == 0) p.wsum[(size_t)b * p.n_chunks + c] = total;
 }
 
 __global__ void __launch_bounds__(kAccThreads) accept_pick_kernel(const AcceptParams p) {
     __shared__ double warp_tot[kAccThreads / 32];
     __shared__ double s_prefix, s_target;
     __shared__ int s_chunk, s_tok, s_target_only;
+    extern __shared__ double ws[];   // [n_chunks] chunk weights
+    pdl_wait();
+    pdl_trigger();
     const int b = blockIdx.x, tid = threadIdx.x;
     const RowInfo ri = p.info[b];
     const float *trow = logit_row(p, b, ri.n);
     const float *drow = ri.bonus ? nullptr : logit_row(p, b, p.gamma + 1 + ri.n);
     double *wsum = p.wsum + (size_t)b * p.n_chunks;
     double w[kAccPerThread], total;
-
+    for (int c = tid; c < p.n_chunks; c += kAccThreads) ws[c] = wsum[c];
+    __syncthreads();
     if (tid == 0) {
         double Z = 0.0;
-        for (int c = 0; c < p.n_chunks; ++c) Z += wsum[c];
+        for (int c = 0; c < p.n_chunks; ++c) Z += ws[c];
         s_target_only = ri.bonus || !(Z > 0.0);
-        s_prefix = Z;
     }
     __syncthreads();
     const bool target_only = s_target_only != 0;
@@ -197,25 +260,62 @@ __global__ void __launch_bounds__(kAccThreads) accept_pick_kernel(const AcceptPa
         for (int c = 0; c < p.n_chunks; ++c) {
             double s = chunk_local(trow, drow, c, p.V, ri, true, w);
             block_scan_inclusive(s, warp_tot, &total);
-            if (tid == 0) wsum[c] = total;
+            if (tid == 0) ws[c] = total;
         }
         __syncthreads();
     }
     if (tid == 0) {
         double Z = 0.0;
-        for (int c = 0; c < p.n_chunks; ++c) Z += wsum[c];
+        for (int c = 0; c < p.n_chunks; ++c) Z += ws[c];
         const double target = (double)p.ur[b] * Z;
         double cum = 0.0;
         int chunk = -1;
         for (int c = 0; c < p.n_chunks; ++c) {
-            if (cum + wsum[c] > target) { chunk = c; break; }
-            cum += wsum[c];
+            if (cum + ws[c] > target) { chunk = c; break; }
+            cum += ws[c];
         }
         s_chunk = chunk; s_prefix = cum; s_target = target; s_tok = 0x7fffffff;
     }
     __syncthreads();
     int tok = -1;
-    if (s_chunk >= 0) {
+    if (s_chunk >= 0 && !(target_only && !ri.bonus)) {
+        // the 16-token group: first thread of the chunk whose stored running sum exceeds the target
+        const int c = s_chunk;
+        const double incl = p.tscan[((size_t)b * p.n_chunks + c) * kAccThreads + tid];
+        const bool over = s_prefix + incl > s_target;
+        const unsigned bal = __ballot_sync(0xffffffffu, over);
+        __shared__ int s_first[kAccThreads / 32];
+        if ((tid & 31) == 0) s_first[tid >> 5] = bal ? (tid & ~31) + __ffs(bal) - 1 : 0x7fffffff;
+        __syncthreads();
+        int first = 0x7fffffff;
+        for (int w8 = 0; w8 < kAccThreads / 32; ++w8) first = min(first, s_first[w8]);
+        if (first != 0x7fffffff && tid == first) {
+            // this thread's tokens alone, in order, from the running sum before them
+            const int t0 = c * kAccChunk + tid * kAccPerThread;
+            double run = s_prefix + incl, back = 0.0;
+            double wt[kAccPerThread];
+#pragma unroll
+            for (int e = 0; e < kAccPerThread; ++e) {
+                wt[e] = t0 + e < p.V ? draw_weight(trow, drow, t0 + e, ri, target_only) : 0.0;
+                back += wt[e];
+            }
+            run -= back;
+            int mine = -1;
+#pragma unroll
+            for (int e = 0; e < kAccPerThread; ++e) {
+                run += wt[e];
+                if (mine < 0 && run > s_target) mine = t0 + e;
+            }
+            // rounding may leave the crossing just past the group's end: then its last positive weight
+            if (mine < 0) {
+#pragma unroll
+                for (int e = 0; e < kAccPerThread; ++e) if (wt[e] > 0.0) mine = t0 + e;
+            }
+            s_tok = mine < 0 ? 0x7fffffff : mine;
+        }
+        __syncthreads();
+        if (s_tok != 0x7fffffff) tok = s_tok;
+    } else if (s_chunk >= 0) {
         const int c = s_chunk;
         double s = chunk_local(trow, drow, c, p.V, ri, target_only, w);
         double incl = block_scan_inclusive(s, warp_tot, &total);
@@ -238,15 +338,37 @@ __global__ void __launch_bounds__(kAccThreads) accept_pick_kernel(const AcceptPa
     if (tid == 0) p.out[(size_t)b * (p.gamma + 1) + ri.n] = tok;
 }
 
-struct AcceptWs { size_t stats_off, wsum_off, info_off, total; int n_chunks; };
+struct AcceptWs { size_t stats_off, wsum_off, info_off, tscan_off, total; int n_chunks; };
 static AcceptWs accept_ws(int B, int gamma, int V) {
     AcceptWs w;
     w.n_chunks = ceil_div(V, kAccChunk);
     w.stats_off = kWsHeaderBytes;
     w.wsum_off = w.stats_off + align_up((size_t)B * (2 * gamma + 1) * w.n_chunks * sizeof(double2), 256);
     w.info_off = w.wsum_off + align_up((size_t)B * w.n_chunks * sizeof(double), 256);
-    w.total = w.info_off + align_up((size_t)B * sizeof(RowInfo), 256);
+    w.tscan_off = w.info_off + align_up((size_t)B * sizeof(RowInfo), 256);
+    w.total = w.tscan_off + align_up((size_t)B * w.n_chunks * kAccThreads * sizeof(double), 256);
     return w;
+}
+
+// The three kernels, launched with programmatic stream serialization (each one waits before it reads).
+static int32_t launch_accept(const AcceptParams &p, cudaStream_t s) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kAccThreads);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3((unsigned)p.n_chunks, (unsigned)(2 * p.gamma + 1), (unsigned)p.B);
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_stats_kernel, p));
+    cfg.gridDim = dim3((unsigned)p.n_chunks, (unsigned)p.B);
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_weigh_kernel, p));
+    cfg.gridDim = dim3((unsigned)p.B);
+    cfg.dynamicSmemBytes = (size_t)p.n_chunks * sizeof(double);
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_pick_kernel, p));
+    count_launches(3);
+    return HIPPO_OK;
 }
 
 }  // namespace hippo
@@ -281,15 +403,10 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
     p.stats = (double2 *)((char *)workspace + w.stats_off);
     p.wsum = (double *)((char *)workspace + w.wsum_off);
     p.info = (RowInfo *)((char *)workspace + w.info_off);
+    p.tscan = (double *)((char *)workspace + w.tscan_off);
     p.B = batch; p.gamma = gamma; p.V = vocab; p.n_chunks = w.n_chunks;
     cudaStream_t s = (cudaStream_t)stream;
-    accept_stats_kernel<<<dim3(w.n_chunks, 2 * gamma + 1, batch), kAccThreads, 0, s>>>(p);
-    accept_decide_kernel<<<batch, kAccThreads, (2 * gamma + 1) * 2 * sizeof(double), s>>>(p);
-    accept_wsum_kernel<<<dim3(w.n_chunks, batch), kAccThreads, 0, s>>>(p);
-    accept_pick_kernel<<<batch, kAccThreads, 0, s>>>(p);
-    count_launches(4);
-    HIPPO_CUDA_TRY(cudaGetLastError());
-    return HIPPO_OK;
+    return launch_accept(p, s);
 }
 
 }  // extern "C"
@@ -359,13 +476,8 @@ extern "C" int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vo
     p.stats = (double2 *)((char *)scratch + w.stats_off);
     p.wsum = (double *)((char *)scratch + w.wsum_off);
     p.info = (RowInfo *)((char *)scratch + w.info_off);
+    p.tscan = (double *)((char *)scratch + w.tscan_off);
     p.B = batch; p.gamma = gamma; p.V = vocab; p.n_chunks = w.n_chunks;
     cudaStream_t s = (cudaStream_t)stream;
-    accept_stats_kernel<<<dim3(w.n_chunks, 2 * gamma + 1, batch), kAccThreads, 0, s>>>(p);
-    accept_decide_kernel<<<batch, kAccThreads, (2 * gamma + 1) * 2 * sizeof(double), s>>>(p);
-    accept_wsum_kernel<<<dim3(w.n_chunks, batch), kAccThreads, 0, s>>>(p);
-    accept_pick_kernel<<<batch, kAccThreads, 0, s>>>(p);
-    count_launches(4);
-    HIPPO_CUDA_TRY(cudaGetLastError());
-    return HIPPO_OK;
+    return launch_accept(p, s);
 }

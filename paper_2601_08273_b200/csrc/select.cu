@@ -63,6 +63,19 @@ __device__ __forceinline__ int find_seq(const int *off, int n, int x) {  // larg
 }
 
 // ---- norms and the dot product with the same cell of the next frame ------------------------------------------
+template <typename T> __device__ __forceinline__ void load8(const T *p, double *v);
+template <> __device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16 *p, double *v) {
+    const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); v[2 * i] = (double)f.x; v[2 * i + 1] = (double)f.y; }
+}
+template <> __device__ __forceinline__ void load8<float>(const float *p, double *v) {
+    const float4 a = __ldg(reinterpret_cast<const float4 *>(p)), c = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+}
+
+// One warp per token; a lane takes 8 consecutive elements per step (embed_dim is a multiple of 8).
 template <typename T>
 __global__ void __launch_bounds__(256) select_dots_kernel(const SelectParams p) {
     const int total = p.seq_off[p.batch];
@@ -75,10 +88,15 @@ __global__ void __launch_bounds__(256) select_dots_kernel(const SelectParams p) 
     const bool has_next = j + p.tpf < p.seq_off[b + 1];
     const size_t c = a + (size_t)p.tpf * p.d;
     double n2 = 0.0, td = 0.0;
-    for (int i = lane; i < p.d; i += 32) {
-        const double x = ld_as_double(E, a + i);
-        n2 = fma(x, x, n2);
-        if (has_next) td = fma(x, ld_as_double(E, c + i), td);
+    for (int i = lane * 8; i < p.d; i += 256) {
+        double x[8], y[8];
+        load8(E + a + i, x);
+        if (has_next) load8(E + c + i, y);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            n2 = fma(x[e], x[e], n2);
+            if (has_next) td = fma(x[e], y[e], td);
+        }
     }
     n2 = warp_sum(n2);
     td = warp_sum(td);
@@ -86,8 +104,48 @@ __global__ void __launch_bounds__(256) select_dots_kernel(const SelectParams p) 
 }
 
 // ---- spatial score: one CTA per crop ---------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(256) select_spatial_kernel(const SelectParams p) {
+// Gram matrix of the crop's (at most 25, in general crop_h*crop_w <= 32) embeddings in fp64.  The embedding dimension is
+// walked in chunks of 128: a chunk of every token of the crop is converted to fp64 once and staged in shared memory
+// (double buffered; the next chunk's global loads are in flight during the arithmetic), then thread (block, slice)
+// accumulates a 5 x 5 block of token pairs over 8 of the 128 dimensions: 10 shared-memory loads feed 25 fused
+// multiply-adds.  The 16 slices of a block are summed by warp shuffles at the end.
+constexpr int kSpaChunk = 128;             // embedding dimensions per staged chunk
+constexpr int kSpaGroup = 5;               // tokens per register-block side
+constexpr int kSpaSlices = 16;             // threads per block of pairs, 8 dimensions each
+// Shape of the kernel for crops of up to NG groups of five tokens: NG = 5 (the paper's 5 x 5 crop, 256 threads, two
+// CTAs per SM) or NG = 7 (up to 32 tokens, 512 threads).
+template <int NG> struct SpaShape {
+    static constexpr int kBlocks = NG * (NG + 1) / 2;                  // upper triangle incl. diagonal
+    static constexpr int kThreads = ((kBlocks * kSpaSlices + 255) / 256) * 256;
+    static constexpr int kRows = NG * kSpaGroup;                       // staged rows (padding rows are zero)
+    static constexpr size_t kSmemBytes = 2 * (size_t)kRows * kSpaChunk * sizeof(double);
+};
+
+template <typename T> struct Chunk8;   // eight consecutive elements of an embedding row
+template <> struct Chunk8<__nv_bfloat16> {
+    uint4 v;
+    __device__ __forceinline__ void load(const __nv_bfloat16 *p) { v = __ldg(reinterpret_cast<const uint4 *>(p)); }
+    __device__ __forceinline__ void zero() { v = make_uint4(0, 0, 0, 0); }
+    __device__ __forceinline__ void store(double *dst) const {
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); dst[2 * i] = (double)f.x; dst[2 * i + 1] = (double)f.y; }
+    }
+};
+template <> struct Chunk8<float> {
+    float4 a, b;
+    __device__ __forceinline__ void load(const float *p) { a = __ldg(reinterpret_cast<const float4 *>(p)); b = __ldg(reinterpret_cast<const float4 *>(p) + 1); }
+    __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
+    __device__ __forceinline__ void store(double *dst) const {
+        dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w; dst[4] = b.x; dst[5] = b.y; dst[6] = b.z; dst[7] = b.w;
+    }
+};
+
+template <typename T, int NG>
+__global__ void __launch_bounds__(SpaShape<NG>::kThreads) select_spatial_kernel(const SelectParams p) {
+    constexpr int kSpaMaxGroups = NG, kSpaMaxBlocks = SpaShape<NG>::kBlocks, kSpaThreads = SpaShape<NG>::kThreads;
+    constexpr int kSpaRows = SpaShape<NG>::kRows;
+    extern __shared__ __align__(16) double stage[];   // [2][kSpaRows][kSpaChunk]
     __shared__ int tok[kMaxCrop];
     __shared__ double S[kMaxCrop][kMaxCrop + 1];
     __shared__ int s_M;
@@ -98,7 +156,8 @@ __global__ void __launch_bounds__(256) select_spatial_kernel(const SelectParams 
     const int n_v = p.seq_off[b + 1] - p.seq_off[b];
     const int nf = min(p.tpf, n_v - f * p.tpf);
     const int y0 = (cr / p.crops_x) * p.crop_h, x0 = (cr % p.crops_x) * p.crop_w;
-    if (threadIdx.x == 0) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    if (tid == 0) {
         int M = 0;
         for (int y = y0; y < y0 + p.crop_h && y < p.grid_h; ++y)
             for (int x = x0; x < x0 + p.crop_w && x < p.grid_w; ++x)
@@ -109,28 +168,97 @@ __global__ void __launch_bounds__(256) select_spatial_kernel(const SelectParams 
     const int M = s_M;
     if (M == 0) return;
     const T *E = (const T *)p.embeds;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    // upper triangle (a < b) of the raw Gram matrix in fp64; norms come from the dots kernel
-    const int n_pairs = M * (M - 1) / 2;
-    for (int pr = warp; pr < n_pairs; pr += nw) {
-        int a = 0, rem = pr;
-        while (rem >= M - 1 - a) { rem -= M - 1 - a; ++a; }
-        const int c = a + 1 + rem;
-        const size_t oa = (size_t)tok[a] * p.d, oc = (size_t)tok[c] * p.d;
-        double acc = 0.0;
-        for (int i = lane; i < p.d; i += 32) acc = fma(ld_as_double(E, oa + i), ld_as_double(E, oc + i), acc);
-        acc = warp_sum(acc);
-        if (lane == 0) {
-            const double na = p.norm2[tok[a]], nc = p.norm2[tok[c]];
-            const double s = (na > 0.0 && nc > 0.0) ? acc / (sqrt(na) * sqrt(nc)) : 0.0;
-            S[a][c] = s;
-            S[c][a] = s;
+    if (M > 1) {
+        const int n_groups = (M + kSpaGroup - 1) / kSpaGroup;
+        // this thread's block of pairs: groups (ga <= gc), and its 8-dimension slice of every chunk
+        const int blk = tid / kSpaSlices, slice = tid % kSpaSlices;
+        int ga = 0, gc = 0;
+        {
+            int rem = blk;
+            while (ga < kSpaMaxGroups && rem >= kSpaMaxGroups - ga) { rem -= kSpaMaxGroups - ga; ++ga; }
+            gc = ga + rem;
         }
+        const bool active = blk < kSpaMaxBlocks && gc < n_groups;
+        double acc[kSpaGroup][kSpaGroup];
+#pragma unroll
+        for (int i = 0; i < kSpaGroup; ++i)
+#pragma unroll
+            for (int j = 0; j < kSpaGroup; ++j) acc[i][j] = 0.0;
+        // staging: item = (row, 8-column piece); rows beyond M are zero
+        const int rows = n_groups * kSpaGroup;
+        const int items = rows * (kSpaChunk / 8);
+        constexpr int kMaxItems = (kSpaRows * (kSpaChunk / 8) + kSpaThreads - 1) / kSpaThreads;
+        Chunk8<T> pre[kMaxItems];
+        auto fetch = [&](int d0) {
+#pragma unroll
+            for (int k = 0; k < kMaxItems; ++k) {
+                const int it = tid + k * kSpaThreads;
+                const int r = it / (kSpaChunk / 8), c8 = it % (kSpaChunk / 8);
+                if (it < items && r < M && d0 + c8 * 8 < p.d) pre[k].load(E + (size_t)tok[r] * p.d + d0 + c8 * 8);
+                else pre[k].zero();
+            }
+        };
+        auto put = [&](int buf) {
+#pragma unroll
+            for (int k = 0; k < kMaxItems; ++k) {
+                const int it = tid + k * kSpaThreads;
+                if (it < items) pre[k].store(stage + ((size_t)buf * kSpaRows + it / (kSpaChunk / 8)) * kSpaChunk + (it % (kSpaChunk / 8)) * 8);
+            }
+        };
+        const int n_chunks = (p.d + kSpaChunk - 1) / kSpaChunk;
+        fetch(0);
+        put(0);
+        __syncthreads();
+        for (int ch = 0; ch < n_chunks; ++ch) {
+            const int buf = ch & 1;
+            if (ch + 1 < n_chunks) fetch((ch + 1) * kSpaChunk);
+            if (active) {
+                const double *ra = stage + ((size_t)buf * kSpaRows + ga * kSpaGroup) * kSpaChunk + slice;
+                const double *rc = stage + ((size_t)buf * kSpaRows + gc * kSpaGroup) * kSpaChunk + slice;
+#pragma unroll
+                for (int k = 0; k < kSpaChunk / kSpaSlices; ++k) {
+                    double va[kSpaGroup], vc[kSpaGroup];
+#pragma unroll
+                    for (int i = 0; i < kSpaGroup; ++i) { va[i] = ra[i * kSpaChunk + k * kSpaSlices]; vc[i] = rc[i * kSpaChunk + k * kSpaSlices]; }
+#pragma unroll
+                    for (int i = 0; i < kSpaGroup; ++i)
+#pragma unroll
+                        for (int j = 0; j < kSpaGroup; ++j) acc[i][j] = fma(va[i], vc[j], acc[i][j]);
+                }
+            }
+            if (ch + 1 < n_chunks) put(buf ^ 1);
+            __syncthreads();
+        }
+        // the 16 slices of a block sit in one half-warp
+#pragma unroll
+        for (int i = 0; i < kSpaGroup; ++i)
+#pragma unroll
+            for (int j = 0; j < kSpaGroup; ++j) {
+                double v = acc[i][j];
+#pragma unroll
+                for (int o = kSpaSlices / 2; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                acc[i][j] = v;
+            }
+        if (active && slice == 0) {
+#pragma unroll
+            for (int i = 0; i < kSpaGroup; ++i)
+#pragma unroll
+                for (int j = 0; j < kSpaGroup; ++j) {
+                    const int ta = ga * kSpaGroup + i, tc = gc * kSpaGroup + j;
+                    if (ta < M && tc < M && ta < tc) {
+                        const double na = p.norm2[tok[ta]], nc = p.norm2[tok[tc]];
+                        const double cs = (na > 0.0 && nc > 0.0) ? acc[i][j] / (sqrt(na) * sqrt(nc)) : 0.0;
+                        S[ta][tc] = cs;
+                        S[tc][ta] = cs;
+                    }
+                }
+        }
+        (void)lane;
     }
-    if (threadIdx.x < M) S[threadIdx.x][threadIdx.x] = 1.0;
+    if (tid < M) S[tid][tid] = 1.0;
     __syncthreads();
-    if (threadIdx.x < M) {
-        const int a = threadIdx.x;
+    if (tid < M) {
+        const int a = tid;
         double mu = 0.0;
         for (int c = 0; c < M; ++c) mu += S[a][c];
         mu /= M;
@@ -213,9 +341,14 @@ __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p)
         __syncthreads();
         const uint32_t prefix = s_prefix;
         const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-        for (int i = tid; i < n; i += blockDim.x) {
-            const uint32_t key = order_key(score[i]);
-            if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        // scores cluster in a few bins: lanes that hit the same bin elect one of them to add their count
+        for (int i0 = 0; i0 < n; i0 += blockDim.x) {
+            const int i = i0 + tid;
+            const uint32_t key = i < n ? order_key(score[i]) : 0u;
+            const bool in = i < n && (key & himask) == prefix;
+            const uint32_t bin = in ? (key >> shift) & 255u : 256u + (uint32_t)lane;   // outsiders match nobody
+            const unsigned peers = __match_any_sync(0xffffffffu, bin);
+            if (in && (int)(__ffs(peers) - 1) == lane) atomicAdd(&hist[bin], __popc(peers));
         }
         __syncthreads();
         if (tid == 0) {
@@ -338,8 +471,21 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
     }
     if (score_mask & HIPPO_SCORE_SPA) {
         dim3 g2((unsigned)(frames * p.crops_y * p.crops_x));
-        if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float><<<g2, 256, 0, s>>>(p);
-        else select_spatial_kernel<__nv_bfloat16><<<g2, 256, 0, s>>>(p);
+        static bool spa_attr = false;
+        if (!spa_attr) {
+            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<float, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<5>::kSmemBytes));
+            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<__nv_bfloat16, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<5>::kSmemBytes));
+            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<float, 7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<7>::kSmemBytes));
+            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<__nv_bfloat16, 7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<7>::kSmemBytes));
+            spa_attr = true;
+        }
+        if (crop_h * crop_w <= 25) {
+            if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float, 5><<<g2, SpaShape<5>::kThreads, SpaShape<5>::kSmemBytes, s>>>(p);
+            else select_spatial_kernel<__nv_bfloat16, 5><<<g2, SpaShape<5>::kThreads, SpaShape<5>::kSmemBytes, s>>>(p);
+        } else {
+            if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float, 7><<<g2, SpaShape<7>::kThreads, SpaShape<7>::kSmemBytes, s>>>(p);
+            else select_spatial_kernel<__nv_bfloat16, 7><<<g2, SpaShape<7>::kThreads, SpaShape<7>::kSmemBytes, s>>>(p);
+        }
         count_launches(1);
     }
     const int fuse_threads = ((p.tpf + 31) / 32) * 32;

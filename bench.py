@@ -196,7 +196,7 @@ def try_graph(fn, torch):
 
 
 def kernel_sweep(cfg, torch, hb, HippoStep, peak, passes=3, max_gb=24.0):
-    """Verify-only and gather-only timings of one configuration (distinct KV buffers per layer)."""
+    """Per-call timings and the whole step of one configuration (distinct KV buffers per layer)."""
     from paper_2601_08273_b200 import workloads as W
     per_layer = sum(n + cfg.n_text + cfg.gamma + 1 for n in W.visual_lengths(cfg)) * 2 * cfg.tgt_kv_heads * cfg.tgt_head_dim * 2
     layers = max(1, min(cfg.tgt_layers, int(max_gb * 1e9 / per_layer)))
@@ -219,6 +219,19 @@ def kernel_sweep(cfg, torch, hb, HippoStep, peak, passes=3, max_gb=24.0):
                 "gather_gbps": st.gather_bytes() / gms / 1e6, "gather_frac_of_measured_peak": st.gather_bytes() / gms / 1e6 / peak})
     sms = timed(lambda: st.select(cur), 3, cur, torch) / 3
     out.update({"select_us": sms * 1e3, "select_embed_mb": st.select_bytes() / 1e6})
+    dreplay = try_graph(lambda: st.draft(torch.cuda.current_stream()), torch)
+    drun = dreplay if dreplay is not None else (lambda: st.draft(cur))
+    drun()
+    dms = timed(drun, passes, cur, torch) / (passes * cfg.gamma * st.Ld)
+    out.update({"draft_us_per_call": dms * 1e3, "draft_kv_mb_per_call": st.draft_kv_bytes_per_call(cfg.gamma // 2) / 1e6})
+    st.accept(cur)
+    out["accept_us"] = timed(lambda: st.accept(cur), 10, cur, torch) / 10 * 1e3
+    # the whole step: select -> gather -> (draft || verify on two streams) -> accept, all target layers if they fit
+    st.run()
+    torch.cuda.synchronize()
+    out["step_ms"] = timed(st.run, passes, cur, torch) / passes
+    out["step_target_layers"] = layers
+    out["step_draft_layers"] = st.Ld
     del st
     torch.cuda.empty_cache()
     return out
@@ -348,7 +361,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_extra:
         del st
         torch.cuda.empty_cache()
-        for ci in (2, 4):
+        for ci in (2, 3, 4):
             try:
                 extra.append(kernel_sweep(W.CONFIGS[ci], torch, hb, HippoStep, peak))
             except Exception as e:  # noqa: BLE001
@@ -406,7 +419,7 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="index into the five configurations (default 1: 7B-class single video)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--no-extra", action="store_true", help="skip the verify/gather sweeps of the 32k and 64k configurations")
+    ap.add_argument("--no-extra", action="store_true", help="skip the per-call timings and whole-step times of the other configurations (c2, c3, c4)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -4,10 +4,13 @@
 // draft keeps only the chosen visual tokens plus the always-kept positions.  A pure copy, bound by HBM bandwidth:
 // per kept token and layer 2 * n_kv_heads * head_dim elements are read and written once.
 //
-// One work item moves 16 bytes; a thread takes four items per round, all four loads issued before the first store.
-// Items are ordered (chunk within row, destination token, head) inside a (layer, K|V) plane given by blockIdx.y, so
-// that consecutive threads write consecutive addresses of one destination (page, head) block; reads are whole rows of
-// head_dim elements (128 B for head_dim 64 bf16) scattered over the source pages.  Index arithmetic is 32-bit.
+// One work item is a 16-byte piece of one kept row: (chunk within row, destination token, head).  Its offsets inside a
+// (layer, K|V) plane are the same for every plane - the page tables are shared by all layers - so a thread resolves
+// its item once (keep index, source and destination page) and then copies that piece in plane after plane, eight
+// loads in flight before the first store.  blockIdx.y splits the planes into groups when there are too few items to
+// fill the machine.  Items are ordered so that consecutive threads write consecutive addresses of one destination
+// (page, head) block; reads are whole rows of head_dim elements (128 B for head_dim 64 bf16) scattered over the
+// source pages.
 #include "common.cuh"
 
 namespace hippo {
@@ -17,49 +20,45 @@ struct GatherParams {
     char *dst_k, *dst_v;
     const int32_t *src_table, *dst_table, *keep_idx, *keep_offsets;
     size_t src_layer_stride, dst_layer_stride;
-    int n_layers, batch, total_keep, n_kv_heads, row_chunks, src_mpps, dst_mpps;
+    int n_layers, batch, total_keep, n_kv_heads, row_chunks, src_mpps, dst_mpps, planes_per_group;
 };
 
 constexpr int kGatherThreads = 256;
-constexpr int kGatherUnroll = 4;
+constexpr int kGatherUnroll = 8;
 
 __global__ void __launch_bounds__(kGatherThreads) gather_kv_kernel(const GatherParams p) {
     const uint32_t per_plane = (uint32_t)p.total_keep * (uint32_t)p.n_kv_heads * (uint32_t)p.row_chunks;
-    const int l = blockIdx.y >> 1, is_v = blockIdx.y & 1;
-    const char *src = (is_v ? p.src_v : p.src_k) + (size_t)l * p.src_layer_stride;
-    char *dst = (is_v ? p.dst_v : p.dst_k) + (size_t)l * p.dst_layer_stride;
-    const uint32_t row_bytes = (uint32_t)p.row_chunks * 16u;
-    const uint32_t stride = gridDim.x * kGatherThreads;
-    for (uint32_t w0 = blockIdx.x * kGatherThreads + threadIdx.x; w0 < per_plane; w0 += stride * kGatherUnroll) {
-        size_t so[kGatherUnroll], dof[kGatherUnroll];
-        bool live[kGatherUnroll];
-#pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u) {
-            const uint32_t w = w0 + u * stride;
-            live[u] = w < per_plane;
-            const uint32_t x = live[u] ? w : 0u;
-            const uint32_t c = x % (uint32_t)p.row_chunks, y = x / (uint32_t)p.row_chunks;
-            const int i = (int)(y % (uint32_t)p.total_keep), h = (int)(y / (uint32_t)p.total_keep);
-            // sequence of flat keep index i: largest b with keep_offsets[b] <= i
-            int lo = 0, hi = p.batch;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (__ldg(p.keep_offsets + mid) <= i) lo = mid; else hi = mid;
-            }
-            const int src_tok = __ldg(p.keep_idx + i);
-            const int dst_tok = i - __ldg(p.keep_offsets + lo);
-            const int sp = page_of(p.src_table, p.src_mpps, lo, src_tok / kPageSize);
-            const int dp = page_of(p.dst_table, p.dst_mpps, lo, dst_tok / kPageSize);
-            so[u] = (((size_t)sp * p.n_kv_heads + h) * kPageSize + (src_tok % kPageSize)) * row_bytes + c * 16u;
-            dof[u] = (((size_t)dp * p.n_kv_heads + h) * kPageSize + (dst_tok % kPageSize)) * row_bytes + c * 16u;
-        }
+    const uint32_t x = blockIdx.x * kGatherThreads + threadIdx.x;
+    if (x >= per_plane) return;
+    const uint32_t c = x % (uint32_t)p.row_chunks, y = x / (uint32_t)p.row_chunks;
+    const int i = (int)(y % (uint32_t)p.total_keep), h = (int)(y / (uint32_t)p.total_keep);
+    // sequence of flat keep index i: largest b with keep_offsets[b] <= i
+    int lo = 0, hi = p.batch;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(p.keep_offsets + mid) <= i) lo = mid; else hi = mid;
+    }
+    const int src_tok = __ldg(p.keep_idx + i);
+    const int dst_tok = i - __ldg(p.keep_offsets + lo);
+    const int sp = page_of(p.src_table, p.src_mpps, lo, src_tok / kPageSize);
+    const int dp = page_of(p.dst_table, p.dst_mpps, lo, dst_tok / kPageSize);
+    const size_t row_bytes = (size_t)p.row_chunks * 16;
+    const size_t so = (((size_t)sp * p.n_kv_heads + h) * kPageSize + (src_tok % kPageSize)) * row_bytes + c * 16u;
+    const size_t dof = (((size_t)dp * p.n_kv_heads + h) * kPageSize + (dst_tok % kPageSize)) * row_bytes + c * 16u;
+    // planes: 2*l + (0 = K, 1 = V)
+    const int pl0 = blockIdx.y * p.planes_per_group, pl1 = min(2 * p.n_layers, pl0 + p.planes_per_group);
+    for (int pl = pl0; pl < pl1; pl += kGatherUnroll) {
         uint4 v[kGatherUnroll];
 #pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u)
-            if (live[u]) v[u] = __ldg(reinterpret_cast<const uint4 *>(src + so[u]));
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int q = pl + u;
+            if (q < pl1) v[u] = __ldg(reinterpret_cast<const uint4 *>(((q & 1) ? p.src_v : p.src_k) + (size_t)(q >> 1) * p.src_layer_stride + so));
+        }
 #pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u)
-            if (live[u]) *reinterpret_cast<uint4 *>(dst + dof[u]) = v[u];
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int q = pl + u;
+            if (q < pl1) *reinterpret_cast<uint4 *>(((q & 1) ? p.dst_v : p.dst_k) + (size_t)(q >> 1) * p.dst_layer_stride + dof) = v[u];
+        }
     }
 }
 
@@ -109,12 +108,15 @@ extern "C" int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src
     const long long per_plane = (long long)total_keep * p.n_kv_heads * p.row_chunks;
     if (per_plane > 0x7fffffffLL) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_gather_kv: more than 2^31 16-byte items per layer");
     if (2 * n_layers > 65535) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_gather_kv: too many layers for one launch");
-    // blocks per (layer, K|V) plane: enough rounds of kGatherUnroll items per thread, at most ~16 blocks per SM in total
-    long long bx = (per_plane + kGatherThreads * kGatherUnroll - 1) / (kGatherThreads * kGatherUnroll);
-    const long long cap = (long long)kNumSMs * 16 / (2 * n_layers) + 1;
-    if (bx > cap) bx = cap;
-    if (bx < 1) bx = 1;
-    gather_kv_kernel<<<dim3((unsigned)bx, (unsigned)(2 * n_layers)), kGatherThreads, 0, (cudaStream_t)stream>>>(p);
+    // plane groups: all planes in one thread when the items alone fill the machine (8 blocks per SM), else split
+    const long long bx = (per_plane + kGatherThreads - 1) / kGatherThreads;
+    long long gy = ((long long)kNumSMs * 8 + bx - 1) / bx;
+    if (gy > 2 * n_layers) gy = 2 * n_layers;
+    if (gy < 1) gy = 1;
+    p.planes_per_group = (int)((2 * n_layers + gy - 1) / gy);
+    gy = (2 * n_layers + p.planes_per_group - 1) / p.planes_per_group;
+    if (bx > 0x7fffffffLL || gy > 65535) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_gather_kv: grid too large");
+    gather_kv_kernel<<<dim3((unsigned)bx, (unsigned)gy), kGatherThreads, 0, (cudaStream_t)stream>>>(p);
     count_launches(1);
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;

@@ -183,6 +183,7 @@ struct TcShared {
     int limit[kMaxRows];        // last visible key of each packed row
     int rowoff[kMaxRows];       // (b*q_len + t)*H_q + h of each packed row, -1 for padding rows
     int tile_prefix[kTcMaxBatch + 1];  // only [0, batch] used
+    int kvlen[kTcMaxBatch];            // kv_len, read once
     // unit-aligned split
     int sum_base;
     uint32_t rem[kMaxAlignedUnits];
@@ -277,7 +278,11 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         else if (tid == nb + 10) mbar_init(smem_u32(&sh->drain), 1);
         else if (tid == nb + 11) { sh->abort = 0; sh->sum_base = 0; }
         // tiles per sequence, then an exclusive prefix
-        for (int b = tid; b < B; b += kTcThreads) sh->tile_prefix[b + 1] = seq_tiles(p.kv_len[b], p.q_len);
+        for (int b = tid; b < B; b += kTcThreads) {
+            const int kvl = p.kv_len[b];
+            sh->kvlen[b] = kvl;
+            sh->tile_prefix[b + 1] = seq_tiles(kvl, p.q_len);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid == 32) {
@@ -410,7 +415,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 locate(t, b, hk, tile);
                 const int nt = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
                 const int n = (int)min((long long)(nt - tile), t_end - t);
-                const int n_pages_seq = (p.kv_len[b] + kPageSize - 1) / kPageSize;
+                const int n_pages_seq = (sh->kvlen[b] + kPageSize - 1) / kPageSize;
                 for (int i = 0; i < n && ok; ++i) {
                     const int pg0 = 2 * (tile + i);
                     const int np = min(2, n_pages_seq - pg0);        // the last tile of a sequence may hold one page
@@ -534,7 +539,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             locate(t, b, hk, tile);
             const int nt = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
             const int n = (int)min((long long)(nt - tile), t_end - t);
-            const int kvl = p.kv_len[b];
+            const int kvl = sh->kvlen[b];
             const bool whole_unit = (tile == 0 && n == nt);
             // ---- per-segment tables and Q -> shared memory (after the previous segment's QK MMAs are done)
             if (seg > 0) ok = W.wait(&sh->q_free, (seg - 1) & 1, 7) && ok;
@@ -737,27 +742,58 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                                         : p.partials + (size_t)(slot_bias * unit + blockIdx.x) * slot_float_count(R, D);
                 const int Rpad = slot_rows_padded(R);
                 __nv_bfloat16 *og = (__nv_bfloat16 *)p.out;
-                for (int c = c_first; c < Rp; c += 32) {
-                    float ov[16];
-                    tmem_ld16(tmem + lane_addr + col_o + c, ov);
-                    tmem_wait_ld();
-                    if (d_active && ok) {
+                const bool direct = whole_unit && !clustered;
+                // per row, by one thread: lse or the partial's (m, l); fscale becomes the factor of the row's outputs
+                if (st < Rp) {
+                    const int r = st;
+                    const float l = sh->fscale[r];
+                    const float m_ref = -sh->mneg[r];   // -inf while nothing was visible
+                    float factor = 0.f;
+                    if (r < R && ok) {
+                        if (direct) {
+                            factor = l > 0.f ? 1.f / l : 0.f;
+                            if (p.lse) p.lse[sh->rowoff[r]] = l > 0.f ? m_ref * kLn2 + logf(l) : -INFINITY;
+                        } else {
+                            factor = (m_ref == -INFINITY) ? 0.f : 1.f;
+                            slot[r] = (m_ref == -INFINITY) ? -INFINITY : m_ref * kLn2;   // natural-log domain for the combine
+                            slot[Rpad + r] = (m_ref == -INFINITY) ? 0.f : l;
+                        }
+                    }
+                    sh->fscale[r] = factor;
+                }
+                softmax_bar_sync();
+                // the outputs: straight-line body, predicated stores
+                const bool store_ok = d_active && ok;
+                if (direct) {
+                    for (int c = c_first; c < Rp; c += 32) {
+                        float ov[16];
+                        tmem_ld16(tmem + lane_addr + col_o + c, ov);
+                        tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const int r = c + e;
-                            if (r < R) {
-                                const float l = sh->fscale[r];
-                                const float m_ref = -sh->mneg[r];   // -inf while nothing was visible
-                                if (whole_unit && !clustered) {
-                                    og[(size_t)sh->rowoff[r] * D + d] = __float2bfloat16_rn(l > 0.f ? ov[e] / l : 0.f);
-                                    if (p.lse && d == (r & (D - 1))) p.lse[sh->rowoff[r]] = l > 0.f ? m_ref * kLn2 + logf(l) : -INFINITY;
-                                } else {
-                                    slot[2 * Rpad + (size_t)r * D + d] = (m_ref == -INFINITY) ? 0.f : ov[e];
-                                    if (d == (r & (D - 1))) {
-                                        slot[r] = (m_ref == -INFINITY) ? -INFINITY : m_ref * kLn2;   // natural-log domain for the combine
-                                        slot[Rpad + r] = (m_ref == -INFINITY) ? 0.f : l;
-                                    }
-                                }
+                        for (int e4 = 0; e4 < 4; ++e4) {
+                            const float4 f = *reinterpret_cast<const float4 *>(&sh->fscale[c + 4 * e4]);
+                            const int4 ro = *reinterpret_cast<const int4 *>(&sh->rowoff[c + 4 * e4]);
+                            const float fv[4] = {f.x, f.y, f.z, f.w};
+                            const int rv4[4] = {ro.x, ro.y, ro.z, ro.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (store_ok && rv4[e] >= 0) og[(size_t)rv4[e] * D + d] = __float2bfloat16_rn(ov[4 * e4 + e] * fv[e]);
+                        }
+                    }
+                } else {
+                    float *so = slot + 2 * Rpad + d;
+                    for (int c = c_first; c < Rp; c += 32) {
+                        float ov[16];
+                        tmem_ld16(tmem + lane_addr + col_o + c, ov);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e4 = 0; e4 < 4; ++e4) {
+                            const float4 f = *reinterpret_cast<const float4 *>(&sh->fscale[c + 4 * e4]);
+                            const float fv[4] = {f.x, f.y, f.z, f.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int r = c + 4 * e4 + e;
+                                if (store_ok && r < R) so[(size_t)r * D] = fv[e] == 0.f ? 0.f : ov[4 * e4 + e];
                             }
                         }
                     }

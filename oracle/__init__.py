@@ -151,3 +151,18 @@ def accept(target_logits, draft_logits, draft_tokens, u_accept, u_resample):
     if rc != 0:
         raise ValueError("oracle_accept rc=%d" % rc)
     return n, out, ma, mc
+
+
+def accept_greedy(target_logits, draft_tokens):
+    """Greedy verification: keep draft tokens while they equal the arg-max of the target row, then emit the
+    target's arg-max.  Returns (n_accepted [B], out_tokens [B][gamma+1])."""
+    tl = _f32(target_logits)
+    B, g1, V = tl.shape
+    g = g1 - 1
+    x = _i32(draft_tokens).reshape(B, g)
+    n = np.empty(B, dtype=np.int32)
+    out = np.empty((B, g + 1), dtype=np.int32)
+    rc = _load().oracle_accept_greedy(B, g, V, _p(tl), _p(x), _p(n), _p(out))
+    if rc != 0:
+        raise ValueError("oracle_accept_greedy rc=%d" % rc)
+    return n, out

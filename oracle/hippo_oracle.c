@@ -376,3 +376,31 @@ int oracle_accept(int B, int gamma, int V, const float *target_logits, const flo
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Greedy verification: the decoding mode of the paper's experiments (Appendix "More Details of
+ * Experiment Setups": answers are generated "following greedy decoding").  With greedy decoding the
+ * target's token at a position is the arg-max of its logit row, so a draft token is kept iff it
+ * equals that arg-max; at the first mismatch n the target's own arg-max is emitted instead, and if all
+ * gamma tokens match, the arg-max of the bonus row gamma.  Ties: the lowest token id.  No uniforms.
+ * ---------------------------------------------------------------------------------------------- */
+int oracle_accept_greedy(int B, int gamma, int V, const float *target_logits, const int32_t *draft_tokens,
+                         int32_t *n_accepted, int32_t *out_tokens) {
+    if (B <= 0 || gamma < 0 || V <= 0) return -1;
+    for (int b = 0; b < B; ++b) {
+        const float *tl = target_logits + (size_t)b * (gamma + 1) * V;
+        int32_t *out = out_tokens + (size_t)b * (gamma + 1);
+        for (int j = 0; j <= gamma; ++j) out[j] = -1;
+        int n = 0;
+        for (;;) {
+            const float *row = tl + (size_t)n * V;
+            int best = 0;
+            for (int t = 1; t < V; ++t) if (row[t] > row[best]) best = t;
+            if (n < gamma && draft_tokens[(size_t)b * gamma + n] == best) { out[n] = best; ++n; continue; }
+            out[n] = best;
+            break;
+        }
+        n_accepted[b] = n;
+    }
+    return 0;
+}

@@ -174,3 +174,53 @@ def test_resample_sweep_reproduces_residual_cdf():
     toks = np.array([run1(tl, dl, [x], [0.9999999], u)[1][0] for u in us])
     np.testing.assert_allclose(np.bincount(toks, minlength=V) / 2000, w / w.sum(), atol=1.5e-3)
     assert w[x] == 0 and not np.any(toks == x)
+
+
+# ---- greedy verification (the decoding mode of the paper's experiments) ---------------------------------------------
+
+def test_greedy_matches_library_argmax_and_hand_cases():
+    rng = np.random.default_rng(5)
+    B, g, V = 6, 4, 37
+    tl = rng.standard_normal((B, g + 1, V)).astype(np.float32)
+    am = tl.argmax(axis=-1).astype(np.int32)                 # numpy's arg-max: first maximum, an independent routine
+    x = am[:, :g].copy()
+    x[1, 0] = (x[1, 0] + 1) % V                              # first token wrong
+    x[2, 2] = (x[2, 2] + 5) % V                              # third token wrong
+    x[3, 3] = (x[3, 3] + 1) % V                              # last token wrong
+    n, out = oracle.accept_greedy(tl, x)
+    assert n.tolist() == [4, 0, 2, 3, 4, 4]
+    for b in range(B):
+        k = int(n[b])
+        assert out[b, :k].tolist() == x[b, :k].tolist()      # kept draft tokens
+        assert out[b, k] == am[b, k]                         # the target's own token at the first mismatch / bonus
+        assert (out[b, k + 1:] == -1).all()
+
+
+def test_greedy_ties_take_the_lowest_token_id():
+    tl = np.zeros((1, 2, 9), np.float32)
+    tl[0, 0, [3, 7]] = 2.0                                   # two equal maxima
+    tl[0, 1, [8, 1]] = 5.0
+    n, out = oracle.accept_greedy(tl, np.array([[3]], np.int32))
+    assert n.tolist() == [1] and out.tolist() == [[3, 1]]
+    n, out = oracle.accept_greedy(tl, np.array([[7]], np.int32))      # 7 ties with 3 but is not the arg-max
+    assert n.tolist() == [0] and out.tolist() == [[3, -1]]
+
+
+def test_greedy_is_the_zero_temperature_limit_of_the_sampling_rule():
+    """With logits scaled until both softmaxes are one-hot, Eq. 1 accepts exactly the draft tokens that equal the
+    target's arg-max and the residual puts all its mass on that arg-max: the sampling oracle (pinned above by the
+    losslessness identity) and the greedy oracle must agree for every uniform."""
+    rng = np.random.default_rng(11)
+    B, g, V = 40, 5, 23
+    tl = rng.standard_normal((B, g + 1, V)).astype(np.float32)
+    dl = tl[:, :g].copy()
+    flip = rng.random((B, g)) < 0.3
+    dl[flip] = rng.standard_normal((int(flip.sum()), V)).astype(np.float32)   # some draft rows disagree
+    x = dl.argmax(axis=-1).astype(np.int32)                 # greedy draft
+    ua = rng.random((B, g), dtype=np.float32)
+    ur = rng.random(B, dtype=np.float32)
+    n_s, out_s, _, _ = oracle.accept(tl * 1e4, dl * 1e4, x, ua, ur)
+    n_g, out_g = oracle.accept_greedy(tl, x)
+    assert n_s.tolist() == n_g.tolist()
+    assert out_s.tolist() == out_g.tolist()
+    assert len(set(n_g.tolist())) >= 3

@@ -48,7 +48,7 @@ typedef enum hippo_status {
 
 typedef enum hippo_dtype { HIPPO_DTYPE_FP32 = 0, HIPPO_DTYPE_BF16 = 1 } hippo_dtype_t;
 
-typedef enum hippo_accept_mode { HIPPO_ACCEPT_SAMPLE = 0 } hippo_accept_mode_t;
+typedef enum hippo_accept_mode { HIPPO_ACCEPT_SAMPLE = 0, HIPPO_ACCEPT_GREEDY = 1 } hippo_accept_mode_t;
 
 /* score_mask bits for hippo_select_tokens (Eq. 7 sums the enabled terms) */
 #define HIPPO_SCORE_ATTN 1u
@@ -176,6 +176,9 @@ int32_t hippo_draft_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, c
  *   n < gamma : emit a token drawn from norm(max(0, P_n - Q_n));   n == gamma : from P_gamma
  *   the draw is the inverse CDF in ascending token id with u_resample[b]: smallest t with cumsum_t > u * total
  * Softmax normalisers, probabilities and CDFs are evaluated in fp64.
+ * mode HIPPO_ACCEPT_GREEDY (the decoding mode of the paper's experiments, Appendix "More Details of Experiment
+ * Setups"): x_{j+1} is kept iff it equals the arg-max of target row j (lowest token id on ties); the emitted token
+ * is the arg-max of target row n.  draft_logits, u_accept and u_resample are not read and may be NULL.
  *   target_logits fp32 [batch][gamma+1][vocab]     draft_logits fp32 [batch][gamma][vocab]
  *   draft_tokens  int32 [batch][gamma] in [0, vocab) u_accept fp32 [batch][gamma]    u_resample fp32 [batch]
  *   n_accepted    out int32 [batch]                 out_tokens out int32 [batch][gamma+1]: accepted draft tokens,

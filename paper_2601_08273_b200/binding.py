@@ -33,6 +33,8 @@ HIPPO_ERR_UNIMPLEMENTED = -6
 HIPPO_DTYPE_FP32 = 0
 HIPPO_DTYPE_BF16 = 1
 HIPPO_SCORE_ALL = 7
+HIPPO_ACCEPT_SAMPLE = 0
+HIPPO_ACCEPT_GREEDY = 1
 PAGE_SIZE = 64
 
 _vp, _i32, _u32, _sz, _f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_float
@@ -238,14 +240,17 @@ def hippo_accept_workspace_bytes(batch: int, gamma: int, vocab: int) -> int:
     return int(lib.hippo_accept_workspace_bytes(batch, gamma, vocab))
 
 
-def hippo_accept(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
-                 u_accept: torch.Tensor, u_resample: torch.Tensor, n_accepted: Optional[torch.Tensor] = None,
-                 out_tokens: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None
+def hippo_accept(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], draft_tokens: torch.Tensor,
+                 u_accept: Optional[torch.Tensor], u_resample: Optional[torch.Tensor],
+                 n_accepted: Optional[torch.Tensor] = None, out_tokens: Optional[torch.Tensor] = None,
+                 workspace: Optional[torch.Tensor] = None, stream=None, mode: int = HIPPO_ACCEPT_SAMPLE
                  ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """mode HIPPO_ACCEPT_SAMPLE: Eq. 1 with residual resampling; HIPPO_ACCEPT_GREEDY: arg-max matching (draft_logits
+    and the uniforms may be None)."""
     B, g1, V = target_logits.shape
     g = g1 - 1
     for t in (target_logits, draft_logits, u_accept, u_resample):
-        assert t.dtype == torch.float32 and t.is_contiguous()
+        assert t is None or (t.dtype == torch.float32 and t.is_contiguous())
     assert draft_tokens.dtype == torch.int32 and draft_tokens.is_contiguous()
     dev = target_logits.device
     if n_accepted is None:
@@ -255,7 +260,7 @@ def hippo_accept(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_
     if workspace is None:
         workspace = new_workspace(hippo_accept_workspace_bytes(B, g, V), dev)
     _check(lib.hippo_accept(B, g, V, _ptr(target_logits), _ptr(draft_logits) if g else None,
-                            _ptr(draft_tokens) if g else None, _ptr(u_accept) if g else None, _ptr(u_resample), 0,
+                            _ptr(draft_tokens) if g else None, _ptr(u_accept) if g else None, _ptr(u_resample), int(mode),
                             _ptr(n_accepted), _ptr(out_tokens), _ptr(workspace), workspace.numel(), _stream(stream)))
     return n_accepted, out_tokens
 

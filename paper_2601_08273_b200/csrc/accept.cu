@@ -350,6 +350,85 @@ static AcceptWs accept_ws(int B, int gamma, int V) {
     return w;
 }
 
+// ---- greedy verification (the decoding mode of the paper's experiments): keep draft tokens while they equal the
+// arg-max of the target row, then emit the target's arg-max (lowest token id on ties).
+//   argmax  per (sequence, target row, chunk): maximum and its first position -> stats[b][row][chunk] = (max, index)
+//   greedy  per sequence: merge the chunks of every row, compare with the draft tokens, write the outputs
+__global__ void __launch_bounds__(kAccThreads) accept_argmax_kernel(const AcceptParams p) {
+    __shared__ float smax[kAccThreads / 32];
+    __shared__ int sidx[kAccThreads / 32];
+    pdl_wait();
+    pdl_trigger();
+    const int c = blockIdx.x, r = blockIdx.y, b = blockIdx.z, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float *row = logit_row(p, b, r);
+    float m = -INFINITY;
+    int mi = 0x7fffffff;
+#pragma unroll
+    for (int e = 0; e < kAccPerThread; ++e) {
+        const int t = c * kAccChunk + e * kAccThreads + tid;     // ascending in e: a strict '>' keeps the first maximum
+        const float v = t < p.V ? row[t] : -INFINITY;
+        if (v > m || (v == m && t < mi && t < p.V)) { m = v; mi = t; }
+    }
+    for (int o = 16; o; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, mi, o);
+        if (om > m || (om == m && oi < mi)) { m = om; mi = oi; }
+    }
+    if (lane == 0) { smax[warp] = m; sidx[warp] = mi; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < kAccThreads / 32; ++w)
+            if (smax[w] > m || (smax[w] == m && sidx[w] < mi)) { m = smax[w]; mi = sidx[w]; }
+        p.stats[((size_t)b * (2 * p.gamma + 1) + r) * p.n_chunks + c] = make_double2((double)m, (double)mi);
+    }
+}
+
+__global__ void __launch_bounds__(kAccThreads) accept_greedy_kernel(const AcceptParams p) {
+    __shared__ int best[kAccMaxRows];
+    pdl_wait();
+    pdl_trigger();
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_rows = 2 * p.gamma + 1;
+    for (int r = warp; r <= p.gamma; r += kAccThreads / 32) {
+        const double2 *st = p.stats + ((size_t)b * n_rows + r) * p.n_chunks;
+        double m = -INFINITY, mi = 2147483647.0;
+        for (int c = lane; c < p.n_chunks; c += 32)
+            if (st[c].x > m || (st[c].x == m && st[c].y < mi)) { m = st[c].x; mi = st[c].y; }
+        for (int o = 16; o; o >>= 1) {
+            const double om = __shfl_xor_sync(0xffffffffu, m, o), oi = __shfl_xor_sync(0xffffffffu, mi, o);
+            if (om > m || (om == m && oi < mi)) { m = om; mi = oi; }
+        }
+        if (lane == 0) best[r] = (int)mi;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const int32_t *x = p.x + (size_t)b * p.gamma;
+        int32_t *out = p.out + (size_t)b * (p.gamma + 1);
+        int n = 0;
+        while (n < p.gamma && x[n] == best[n]) { out[n] = x[n]; ++n; }
+        out[n] = best[n];
+        for (int j = n + 1; j <= p.gamma; ++j) out[j] = -1;
+        p.n_acc[b] = n;
+    }
+}
+
+static int32_t launch_accept_greedy(const AcceptParams &p, cudaStream_t s) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kAccThreads);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3((unsigned)p.n_chunks, (unsigned)(p.gamma + 1), (unsigned)p.B);
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_argmax_kernel, p));
+    cfg.gridDim = dim3((unsigned)p.B);
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_greedy_kernel, p));
+    count_launches(2);
+    return HIPPO_OK;
+}
+
 // The three kernels, launched with programmatic stream serialization (each one waits before it reads).
 static int32_t launch_accept(const AcceptParams &p, cudaStream_t s) {
     cudaLaunchAttribute attr[1];
@@ -386,10 +465,11 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
                      void *workspace, size_t workspace_bytes, void *stream) {
     using namespace hippo;
     if (batch <= 0 || gamma < 0 || vocab <= 0) return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept: bad sizes");
-    if (mode != HIPPO_ACCEPT_SAMPLE) return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept: mode %d", mode);
-    if (!target_logits || !u_resample || !n_accepted || !out_tokens || !workspace)
+    if (mode != HIPPO_ACCEPT_SAMPLE && mode != HIPPO_ACCEPT_GREEDY) return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept: mode %d", mode);
+    const bool greedy = mode == HIPPO_ACCEPT_GREEDY;
+    if (!target_logits || !n_accepted || !out_tokens || !workspace || (!greedy && !u_resample))
         return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept: null pointer");
-    if (gamma > 0 && (!draft_logits || !draft_tokens || !u_accept))
+    if (gamma > 0 && (!draft_tokens || (!greedy && (!draft_logits || !u_accept))))
         return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept: null draft arrays with gamma > 0");
     if (gamma > 64) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_accept: gamma > 64");
     if ((uintptr_t)workspace & 255) return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept: workspace must be 256-byte aligned");
@@ -406,7 +486,7 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
     p.tscan = (double *)((char *)workspace + w.tscan_off);
     p.B = batch; p.gamma = gamma; p.V = vocab; p.n_chunks = w.n_chunks;
     cudaStream_t s = (cudaStream_t)stream;
-    return launch_accept(p, s);
+    return greedy ? launch_accept_greedy(p, s) : launch_accept(p, s);
 }
 
 }  // extern "C"

@@ -33,7 +33,7 @@ def test_argument_validation_happens_before_any_launch():
     assert lib.hippo_accept(0, 1, 10, None, None, None, None, None, 0, None, None, None, 0, None) == hb.HIPPO_ERR_INVALID_ARG
     assert lib.hippo_accept(1, 1, 10, None, None, None, None, None, 0, None, None, None, 0, None) == hb.HIPPO_ERR_INVALID_ARG
     assert b"null pointer" in lib.hippo_last_error()
-    assert lib.hippo_accept(1, 1, 10, 256, 256, 256, 256, 256, 7, 256, 256, 256, 1 << 20, None) == hb.HIPPO_ERR_UNIMPLEMENTED
+    assert lib.hippo_accept(1, 1, 10, 256, 256, 256, 256, 256, 7, 256, 256, 256, 1 << 20, None) == hb.HIPPO_ERR_UNIMPLEMENTED   # unknown mode
     assert lib.hippo_accept(1, 1, 10, 256, 256, 256, 256, 256, 0, 256, 256, 256, 16, None) == hb.HIPPO_ERR_WORKSPACE_TOO_SMALL
     kv = hb.KVCacheStruct(ctypes.sizeof(hb.KVCacheStruct), hb.HIPPO_DTYPE_BF16, 2, 64, 10, 4, 1024, 2048, None)
     args = lambda **o: [o.get("B", 1), o.get("q_len", 1), o.get("hq", 14), 256, ctypes.byref(kv), 256,

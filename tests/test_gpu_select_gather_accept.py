@@ -219,3 +219,24 @@ def test_accept_odd_vocab_and_gamma0(hb):
     check_accept(hb, W.accept_inputs(cfg, batch=5, gamma=3, vocab=4099, corr_eps=0.5), "V=4099")
     check_accept(hb, W.accept_inputs(cfg, batch=3, gamma=0, vocab=777), "gamma 0")
     check_accept(hb, W.accept_inputs(cfg, batch=3, gamma=1, vocab=3, corr_eps=2.0), "V=3")
+
+
+@pytest.mark.parametrize("ci", [0, 1, 3])
+def test_accept_greedy(hb, ci):
+    """Greedy verification: bit-exact against the oracle; draft tokens = arg-max of draft rows that partly agree."""
+    cfg = W.CONFIGS[ci]
+    B = max(cfg.batch, 6)
+    inp = W.accept_inputs(cfg, batch=B, corr_eps=0.0, sub=5)
+    tl = inp["target_logits"]
+    x = tl[:, :cfg.gamma].argmax(axis=-1).astype(np.int32)
+    rng = np.random.default_rng(ci)
+    wrong = rng.random(x.shape) < 0.25
+    x[wrong] = rng.integers(0, cfg.vocab, size=int(wrong.sum()))
+    x[0] = tl[0, :cfg.gamma].argmax(axis=-1)                 # one sequence accepts everything
+    tl[1, 0, 5] = tl[1, 0, 9] = tl[1, 0].max() + 1.0          # a tie: the lowest id wins
+    n, out = hb.hippo_accept(dev(tl), None, dev(x), None, None, mode=hb.HIPPO_ACCEPT_GREEDY)
+    torch.cuda.synchronize()
+    rn, rout = oracle.accept_greedy(tl, x)
+    np.testing.assert_array_equal(host(n), rn)
+    np.testing.assert_array_equal(host(out), rout)
+    assert rn[0] == cfg.gamma and len(set(rn.tolist())) >= 2

@@ -260,18 +260,14 @@ def run_ours(args):
     st = HippoStep(cfg)
     cur = torch.cuda.current_stream()
 
+    from paper_2601_08273_b200 import replicas
+    dev0 = torch.device("cuda", local)
+
     def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(dev0)
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, dev0)
 
     # warm-up (eager), counting this library's launches per step
     c0 = hb.hippo_launch_count()

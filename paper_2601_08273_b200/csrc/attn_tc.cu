@@ -264,24 +264,72 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     // stream drains; nothing is read or written before that kernel has completed.
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // ---- set-up: barriers, tile prefix, tensor memory
+    // ---- set-up: barriers, tile prefix, CTA split, tensor memory
+    const int U = B * Hkv;
+    const bool clustered = cluster_size > 1;                  // one cluster per unit, merge through shared memory
+    const bool aligned = !clustered && U <= (int)gridDim.x && U <= kMaxAlignedUnits;
+    const bool small_problem = U <= 32;                       // tile prefix and CTA split by warp 0 alone, no block barriers
     {
-        // one barrier per thread: [0, n_slots) full, [n_slots, 2 n_slots) empty, then the fixed ones
-        const int nb = 2 * n_slots;
-        if (tid < nb) mbar_init(smem_u32(tid < n_slots ? &sh->full[tid] : &sh->empty[tid - n_slots]), 1);
-        else if (tid < nb + 2) mbar_init(smem_u32(&sh->s_full[tid - nb]), 1);
-        else if (tid < nb + 4) mbar_init(smem_u32(&sh->s_free[tid - nb - 2]), kSoftmaxThreads);
-        else if (tid < nb + 6) mbar_init(smem_u32(&sh->p_full[tid - nb - 4]), kSoftmaxThreads);
-        else if (tid < nb + 8) mbar_init(smem_u32(&sh->pv_done[tid - nb - 6]), 1);
-        else if (tid == nb + 8) mbar_init(smem_u32(&sh->q_full), kSoftmaxThreads);
-        else if (tid == nb + 9) mbar_init(smem_u32(&sh->q_free), 1);
-        else if (tid == nb + 10) mbar_init(smem_u32(&sh->drain), 1);
-        else if (tid == nb + 11) { sh->abort = 0; sh->sum_base = 0; }
-        // tiles per sequence, then an exclusive prefix
-        for (int b = tid; b < B; b += kTcThreads) {
-            const int kvl = p.kv_len[b];
-            sh->kvlen[b] = kvl;
-            sh->tile_prefix[b + 1] = seq_tiles(kvl, p.q_len);
+        // one barrier per thread of warps 1..: [0, n_slots) full, [n_slots, 2 n_slots) empty, then the fixed ones
+        const int nb = 2 * n_slots, t = tid - 32;
+        if (t < 0) {}
+        else if (t < nb) mbar_init(smem_u32(t < n_slots ? &sh->full[t] : &sh->empty[t - n_slots]), 1);
+        else if (t < nb + 2) mbar_init(smem_u32(&sh->s_full[t - nb]), 1);
+        else if (t < nb + 4) mbar_init(smem_u32(&sh->s_free[t - nb - 2]), kSoftmaxThreads);
+        else if (t < nb + 6) mbar_init(smem_u32(&sh->p_full[t - nb - 4]), kSoftmaxThreads);
+        else if (t < nb + 8) mbar_init(smem_u32(&sh->pv_done[t - nb - 6]), 1);
+        else if (t == nb + 8) mbar_init(smem_u32(&sh->q_full), kSoftmaxThreads);
+        else if (t == nb + 9) mbar_init(smem_u32(&sh->q_free), 1);
+        else if (t == nb + 10) mbar_init(smem_u32(&sh->drain), 1);
+        else if (t == nb + 11) { sh->abort = 0; sh->sum_base = 0; }
+        if (!small_problem) {
+            // tiles per sequence; the exclusive prefix follows the barrier
+            for (int b = tid; b < B; b += kTcThreads) {
+                const int kvl = p.kv_len[b];
+                sh->kvlen[b] = kvl;
+                sh->tile_prefix[b + 1] = seq_tiles(kvl, p.q_len);
+            }
+        } else if (warp == 0) {
+            // lane b: sequence b; lane u: unit u.  Everything by shuffles.
+            const int kvl = lane < B ? p.kv_len[lane] : 0;
+            const int nt = lane < B ? seq_tiles(kvl, p.q_len) : 0;
+            int incl = nt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+            if (lane < B) { sh->kvlen[lane] = kvl; sh->tile_prefix[lane + 1] = incl; }
+            if (lane == 0) sh->tile_prefix[0] = 0;
+            if (aligned) {
+                // CTAs per unit: one each, the others in proportion to the tile counts (largest remainders first)
+                const long long total = (long long)__shfl_sync(0xffffffffu, incl, 31) * Hkv;
+                const int t_src = __shfl_sync(0xffffffffu, nt, lane < U ? lane / Hkv : 0);
+                const int my_tiles = lane < U ? t_src : 0;
+                const bool live = my_tiles > 0;
+                const int spare = (int)gridDim.x - __popc(__ballot_sync(0xffffffffu, live));
+                int base = 0;
+                uint32_t r = 0;
+                if (live) {
+                    const long long num = (long long)spare * my_tiles;
+                    base = (int)(num / total);
+                    r = (uint32_t)(num % total);
+                }
+                int sum_base = base;
+#pragma unroll
+                for (int o = 16; o; o >>= 1) sum_base += __shfl_xor_sync(0xffffffffu, sum_base, o);
+                const int leftover = spare - sum_base;
+                int rank = 0;
+                for (int v = 0; v < U; ++v) {
+                    const uint32_t rv = __shfl_sync(0xffffffffu, r, v);
+                    const int lv = __shfl_sync(0xffffffffu, (int)live, v);
+                    rank += (lv && (rv > r || (rv == r && v < lane))) ? 1 : 0;
+                }
+                const int n = live ? min(my_tiles, 1 + base + (rank < leftover ? 1 : 0)) : 0;
+                int cinc = n;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, cinc, o); if (lane >= o) cinc += v; }
+                if (lane < U) { sh->n_cta[lane] = n; sh->cta_base[lane] = cinc - n; }
+                const int all = __shfl_sync(0xffffffffu, cinc, 31);
+                if (lane == 0) sh->cta_base[U] = all;
+            }
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -295,12 +343,14 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     }
     tc_fence_before();
     __syncthreads();
-    if (tid == 0) {
-        int acc = 0;
-        for (int b = 0; b < B; ++b) { const int n = sh->tile_prefix[b + 1]; sh->tile_prefix[b] = acc; acc += n; }
-        sh->tile_prefix[B] = acc;
+    if (!small_problem) {
+        if (tid == 0) {
+            int acc = 0;
+            for (int b = 0; b < B; ++b) { const int n = sh->tile_prefix[b + 1]; sh->tile_prefix[b] = acc; acc += n; }
+            sh->tile_prefix[B] = acc;
+        }
+        __syncthreads();
     }
-    __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
     const uint32_t col_s = 0, col_o = 2 * Rp, col_l = 3 * Rp;   // S^T[0] | S^T[1] | O^T | partial row sums, Rp columns each
@@ -308,9 +358,6 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     Partition part;
     part.total = (long long)sh->tile_prefix[B] * Hkv;
     part.grid = gridDim.x;
-    const int U = B * Hkv;
-    const bool clustered = cluster_size > 1;                  // one cluster per unit, merge through shared memory
-    const bool aligned = !clustered && U <= (int)gridDim.x && U <= kMaxAlignedUnits;
     long long t_begin = 0, t_end = 0;
     int2 *unit_info = reinterpret_cast<int2 *>(p.counters);   // per unit: first slot, number of contributing CTAs
     if (clustered) {
@@ -321,6 +368,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         t_begin = unit_start + T * i / cluster_size;
         t_end = unit_start + T * (i + 1) / cluster_size;
     } else if (aligned) {
+      if (!small_problem) {
         // CTAs per unit: one each, the others in proportion to the tile counts (largest remainders first)
         const int my_tiles = tid < U ? sh->tile_prefix[tid / Hkv + 1] - sh->tile_prefix[tid / Hkv] : 0;
         const bool live = my_tiles > 0;
@@ -353,6 +401,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             sh->cta_base[U] = acc;
         }
         __syncthreads();
+      }
         if (blockIdx.x == 0 && tid < U) unit_info[tid] = make_int2(sh->cta_base[tid], sh->n_cta[tid]);
         if ((int)blockIdx.x < sh->cta_base[U]) {
             int lo = 0, hi = U;   // largest u with cta_base[u] <= blockIdx.x
@@ -819,7 +868,17 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             for (int r = tid; r < R; r += kTcThreads) { mine[r] = -INFINITY; mine[Rpad + r] = 0.f; }
         }
         cluster_sync_all();
-        if (sh->tile_prefix[b + 1] != sh->tile_prefix[b]) {
+        if (sh->tile_prefix[b + 1] == sh->tile_prefix[b]) {
+            // a sequence shorter than q_len is skipped: its outputs are defined as zero (rows of this unit, by rank 0)
+            if (rank == 0) {
+                for (int x = tid; x < R * D; x += kTcThreads) {
+                    const int r = x / D;
+                    const size_t ro = (size_t)(b * p.q_len + r / G) * p.n_q_heads + hk * G + r % G;
+                    ((__nv_bfloat16 *)p.out)[ro * D + x % D] = __float2bfloat16_rn(0.f);
+                    if (p.lse && x % D == 0) p.lse[ro] = -INFINITY;
+                }
+            }
+        } else {
             // rows r = rank, rank + cluster_size, ... of the unit are merged here, one warp per row
             constexpr int V = D / 32;
             const uint32_t local = smem_u32(mine);
@@ -892,14 +951,14 @@ __global__ void __launch_bounds__(kCombineThreads) attn_tc_combine_kernel(const 
     const int h = row % p.n_q_heads, t = (row / p.n_q_heads) % p.q_len, b = row / (p.n_q_heads * p.q_len);
     const int hk = h / G, r = t * G + (h % G);
     __nv_bfloat16 *out = (__nv_bfloat16 *)p.out + (size_t)row * D;
-    if (seq_tiles(p.kv_len[b], p.q_len) == 0) {
+    const int2 info = reinterpret_cast<const int2 *>(p.counters)[b * Hkv + hk];   // first slot, contributors
+    const int n = info.y;
+    if (n == 0) {   // a sequence shorter than q_len is skipped: its outputs are defined as zero
         if (tid < D) out[tid] = __float2bfloat16_rn(0.f);
         if (p.lse && tid == 0) p.lse[row] = -INFINITY;
         return;
     }
-    const int2 info = reinterpret_cast<const int2 *>(p.counters)[b * Hkv + hk];   // first slot, contributors
-    const int n = info.y;
-    if (n <= 1) return;
+    if (n == 1) return;
     const size_t slot_floats = slot_float_count(R, D);
     const int Rp = slot_rows_padded(R);
     const float *base = p.partials + (size_t)info.x * slot_floats;

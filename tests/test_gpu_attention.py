@@ -113,6 +113,21 @@ def test_short_sequence_is_skipped_and_zeroed(hb):
     assert_close(got[1:], ref, 1e-5)
 
 
+def test_short_sequence_in_a_bf16_batch(hb):
+    """bf16 path, few units (one cluster or one group of CTAs per unit): a sequence shorter than q_len gives zeros."""
+    rng = np.random.default_rng(4)
+    B, q_len, Hq, Hkv, D = 3, 4, 8, 2, 128
+    lens = [700, 3, 260]
+    q = W.round_to_storage(rng.standard_normal((B, q_len, Hq, D)).astype(np.float32), "bf16")
+    k = W.round_to_storage(rng.standard_normal((B, max(lens), Hkv, D)).astype(np.float32), "bf16")
+    v = W.round_to_storage(rng.standard_normal((B, max(lens), Hkv, D)).astype(np.float32), "bf16")
+    for splits in (0, 3):
+        got, lse = run_case(hb, hb.hippo_verify_attention, q, k, v, lens, "bf16", shuffle_seed=2, num_splits=splits)
+        assert np.all(got[1] == 0) and np.all(np.isneginf(lse[1]))
+        ref, _ = oracle.attention(q[[0, 2]], k[[0, 2]], v[[0, 2]], [lens[0], lens[2]])
+        assert_close(got[[0, 2]], ref, TOL["bf16"], "neighbours of a skipped sequence")
+
+
 def sampled_rows(rng, B, q_len, Hq, n):
     rows = {(0, 0, 0), (B - 1, q_len - 1, Hq - 1)}
     while len(rows) < n:

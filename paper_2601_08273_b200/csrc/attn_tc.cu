@@ -170,7 +170,9 @@ struct Partition {
     __device__ __forceinline__ int cta_of(long long t) const { return (int)(((t + 1) * grid - 1) / total); }
 };
 
-__device__ __forceinline__ int seq_tiles(int kvl, int q_len) { return kvl < q_len ? 0 : (kvl + kBlockN - 1) / kBlockN; }
+// The work of a sequence is counted in 64-key pages: CTA ranges begin and end on page boundaries, and a CTA forms its
+// 128-key tiles from consecutive pairs of its pages (the last tile of a range may hold a single page).
+__device__ __forceinline__ int seq_tiles(int kvl, int q_len) { return kvl < q_len ? 0 : (kvl + kPageSize - 1) / kPageSize; }
 
 // ---- shared control block -------------------------------------------------------------------------------------------
 struct TcShared {
@@ -261,8 +263,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
     const int R = p.rows, G = p.group, Hkv = p.n_kv_heads, B = p.batch;
     const Waiter W{sh, p.header};
     // Launched with programmatic stream serialization: the CTAs may be scheduled while the previous kernel of the
-    // stream drains; nothing is read or written before that kernel has completed.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // stream drains.  Barriers and tensor memory are set up meanwhile; global memory is not touched before that
+    // kernel has completed (griddepcontrol.wait below).
 
     // ---- set-up: barriers, tile prefix, CTA split, tensor memory
     const int U = B * Hkv;
@@ -282,6 +284,15 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         else if (t == nb + 9) mbar_init(smem_u32(&sh->q_free), 1);
         else if (t == nb + 10) mbar_init(smem_u32(&sh->drain), 1);
         else if (t == nb + 11) { sh->abort = 0; sh->sum_base = 0; }
+        if (tid == 32) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&v_map) : "memory");
+        }
+        if (warp == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (!small_problem) {
             // tiles per sequence; the exclusive prefix follows the barrier
             for (int b = tid; b < B; b += kTcThreads) {
@@ -332,14 +343,6 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             }
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (tid == 32) {
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&v_map) : "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
@@ -464,10 +467,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 locate(t, b, hk, tile);
                 const int nt = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
                 const int n = (int)min((long long)(nt - tile), t_end - t);
-                const int n_pages_seq = (sh->kvlen[b] + kPageSize - 1) / kPageSize;
-                for (int i = 0; i < n && ok; ++i) {
-                    const int pg0 = 2 * (tile + i);
-                    const int np = min(2, n_pages_seq - pg0);        // the last tile of a sequence may hold one page
+                for (int i = 0; i < n && ok; i += 2) {
+                    const int pg0 = tile + i;
+                    const int np = min(2, n - i);                    // the last tile of a range may hold one page
                     int row[2];
                     for (int q = 0; q < np; ++q)
                         row[q] = (page_of(p.page_table, p.max_pages_per_seq, b, pg0 + q) * Hkv + hk) * kPageSize;
@@ -537,7 +539,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 const int n = (int)min((long long)(nt - tile), t_end - t);
                 ok = W.wait(&sh->q_full, seg & 1, 4);  // Q of this segment is in shared memory
                 const uint32_t it0 = it;
-                for (int i = 0; i < n && ok; ++i, ++it) {
+                for (int i = 0; i < n && ok; i += 2, ++it) {
                     const int j = it & 1;
                     ok = W.wait(&sh->full[rk.slot], rk.phase, 5);
                     if (!ok) break;
@@ -553,9 +555,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                                    qdesc0 + (uint64_t)(c * q_chunk16 + ks * 2), idesc_qk, (c | ks) ? 1u : 0u);
                     tc_commit(smem_u32(&sh->s_full[j]));
                     tc_commit(smem_u32(&sh->empty[rk.slot]));            // K is not needed again
-                    if (i == n - 1) tc_commit(smem_u32(&sh->q_free));    // last QK of the segment: Q may be replaced
+                    if (i + 2 >= n) tc_commit(smem_u32(&sh->q_free));    // last QK of the segment: Q may be replaced
                     rk.advance(n_slots); rk.advance(n_slots);
-                    if (i >= 1) ok = issue_pv(it - 1, it - 1 == it0);    // PV trails QK by one tile
+                    if (i >= 2) ok = issue_pv(it - 1, it - 1 == it0);    // PV trails QK by one tile
                 }
                 if (ok && n >= 1) ok = issue_pv(it - 1, it - 1 == it0);
                 t += n;
@@ -598,7 +600,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                     sh->limit[st] = kvl - p.q_len + tq;
                     sh->rowoff[st] = (b * p.q_len + tq) * p.n_q_heads + hk * G + g;
                 } else {
-                    sh->limit[st] = 0x7fffffff;
+                    sh->limit[st] = 0x7ffffffe;
                     sh->rowoff[st] = -1;
                 }
                 sh->mneg[st] = INFINITY;
@@ -616,18 +618,20 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
 
             const uint32_t it0 = it;
             bool aborted = false;
-            for (int i = 0; i < n; ++i, ++it, rv.advance(n_slots), rv.advance(n_slots)) {
+            for (int i = 0; i < n; i += 2, ++it, rv.advance(n_slots), rv.advance(n_slots)) {
                 const int j = it & 1;
-                const int key0 = (tile + i) * kBlockN;
-                const int key = key0 + kk;
-                const bool tail = key0 + kBlockN > kvl - p.q_len + 1;  // some row needs masking in this tile
+                const int key0 = (tile + i) * kPageSize;
+                const int key_end = min(kvl, key0 + min(2, n - i) * kPageSize);   // first key of the tile that is not there
+                // a key that is not there compares greater than every row's limit
+                const int key = key0 + kk < key_end ? key0 + kk : 0x7fffffff;
+                const bool tail = key0 + kBlockN > kvl - p.q_len + 1 || key0 + kBlockN > key_end;  // some masking in this tile
                 const uint32_t s_addr = tmem + lane_addr + col_s + j * Rp;
-                if (key0 + kBlockN > kvl) {
-                    // rows of V past the end of the sequence may hold anything (also a whole missing second page):
-                    // zero them, 0 * NaN would poison O
+                if (key0 + kBlockN > key_end) {
+                    // rows of V past the end of the sequence or of this CTA's range may hold anything (also a whole
+                    // missing second page): zero them, 0 * NaN would poison O
                     ok = W.wait(&sh->full[rv.slot], rv.phase, 8) && ok;
                     uint8_t *vs = ring + rv.slot * kSlotBytes;
-                    const int first_bad = kvl - key0;
+                    const int first_bad = key_end - key0;
                     for (int x = st; x < (kBlockN - first_bad) * kChunks * 8; x += kSoftmaxThreads) {
                         const int row = first_bad + x / (kChunks * 8), rem = x % (kChunks * 8);
                         *reinterpret_cast<uint4 *>(vs + (row >> 6) * kPageBytes + (rem >> 3) * 8192 + (row & 63) * 128 + ((rem & 7) << 4)) =
@@ -1140,7 +1144,7 @@ int32_t launch_attn_tc(const AttnParams &p, bool draft_policy, cudaStream_t stre
     (void)draft_policy;
     // Upper bound of the tile count from the host-side length bound; the kernel derives the exact partition from
     // kv_len on the device.  The grid never exceeds the bound, so no CTA is started without work to look for.
-    const long long max_tiles = (long long)p.batch * p.n_kv_heads * ceil_div(p.max_kv_len, kBlockN);
+    const long long max_tiles = (long long)p.batch * p.n_kv_heads * ceil_div(p.max_kv_len, kPageSize);
     long long grid = p.num_splits > 0 ? (long long)p.num_splits * p.batch * p.n_kv_heads : kNumSMs;
     if (grid > max_tiles) grid = max_tiles;
     if (grid > kExtraSlots) grid = kExtraSlots;

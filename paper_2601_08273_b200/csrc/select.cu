@@ -323,7 +323,6 @@ __device__ __forceinline__ uint32_t order_key(float x) {  // larger float -> lar
 }
 
 __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p) {
-    __shared__ int hist[256];
     __shared__ int warp_cnt[32];
     __shared__ uint32_t s_prefix;
     __shared__ int s_remaining, s_base_eq, s_base_out;
@@ -333,62 +332,110 @@ __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p)
     if (k <= 0) return;
     const float *score = p.fused + p.seq_off[b];
     int32_t *out = p.kept + p.k_off[b];
-    // radix select: find the key T of the k-th largest element
-    if (tid == 0) { s_prefix = 0; s_remaining = k; }
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        for (int i = tid; i < 256; i += blockDim.x) hist[i] = 0;
-        __syncthreads();
-        const uint32_t prefix = s_prefix;
-        const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-        // scores cluster in a few bins: lanes that hit the same bin elect one of them to add their count
-        for (int i0 = 0; i0 < n; i0 += blockDim.x) {
-            const int i = i0 + tid;
-            const uint32_t key = i < n ? order_key(score[i]) : 0u;
-            const bool in = i < n && (key & himask) == prefix;
-            const uint32_t bin = in ? (key >> shift) & 255u : 256u + (uint32_t)lane;   // outsiders match nobody
-            const unsigned peers = __match_any_sync(0xffffffffu, bin);
-            if (in && (int)(__ffs(peers) - 1) == lane) atomicAdd(&hist[bin], __popc(peers));
+    // The key T of the k-th largest element, two bits at a time from the top: T is the largest value with at least k
+    // keys >= T.  Each thread keeps its keys in registers (up to 32 per thread; longer sequences are read again from
+    // memory), so a step is a few compares and one block-wide sum of three counters.
+    constexpr int kKeysPerThread = 32;
+    __shared__ int warp_cnt3[32][3];
+    __shared__ int s_cnt3[3];
+    uint32_t keys[kKeysPerThread];
+    const bool in_regs = n <= kKeysPerThread * (int)blockDim.x;
+    if (in_regs) {
+#pragma unroll
+        for (int e = 0; e < kKeysPerThread; ++e) {
+            const int i = e * blockDim.x + tid;
+            keys[e] = i < n ? order_key(score[i]) : 0u;   // padding: key 0 is never counted (candidates are > 0)
         }
-        __syncthreads();
-        if (tid == 0) {
-            int rem = s_remaining, bin = 255;
-            for (; bin > 0; --bin) {
-                if (hist[bin] >= rem) break;
-                rem -= hist[bin];
-            }
-            s_prefix = prefix | ((uint32_t)bin << shift);
-            s_remaining = rem;  // how many of the elements inside this bin are still needed
-        }
-        __syncthreads();
     }
+    const int per_thread = (n + (int)blockDim.x - 1) / (int)blockDim.x;
+    // counts of keys >= c1, >= c2, >= c3 over the sequence (candidates are non-zero)
+    auto count3 = [&](uint32_t c1, uint32_t c2, uint32_t c3) {
+        int a1 = 0, a2 = 0, a3 = 0;
+        if (in_regs) {
+#pragma unroll
+            for (int e0 = 0; e0 < kKeysPerThread; e0 += 8) {
+                if (e0 < per_thread) {      // uniform: only the groups of eight that hold keys
+#pragma unroll
+                    for (int e = e0; e < e0 + 8; ++e) {
+                        a1 += keys[e] >= c1 ? 1 : 0; a2 += keys[e] >= c2 ? 1 : 0; a3 += keys[e] >= c3 ? 1 : 0;
+                    }
+                }
+            }
+        } else {
+            for (int i = tid; i < n; i += blockDim.x) {
+                const uint32_t key = order_key(score[i]);
+                a1 += key >= c1 ? 1 : 0; a2 += key >= c2 ? 1 : 0; a3 += key >= c3 ? 1 : 0;
+            }
+        }
+        a1 = __reduce_add_sync(0xffffffffu, a1);
+        a2 = __reduce_add_sync(0xffffffffu, a2);
+        a3 = __reduce_add_sync(0xffffffffu, a3);
+        __syncthreads();                 // the counters of the previous step have been read
+        if (lane == 0) { warp_cnt3[warp][0] = a1; warp_cnt3[warp][1] = a2; warp_cnt3[warp][2] = a3; }
+        __syncthreads();
+        if (warp == 0) {
+            const bool has = lane < (int)(blockDim.x >> 5);
+            int t1 = has ? warp_cnt3[lane][0] : 0, t2 = has ? warp_cnt3[lane][1] : 0, t3 = has ? warp_cnt3[lane][2] : 0;
+            t1 = __reduce_add_sync(0xffffffffu, t1);
+            t2 = __reduce_add_sync(0xffffffffu, t2);
+            t3 = __reduce_add_sync(0xffffffffu, t3);
+            if (lane == 0) { s_cnt3[0] = t1; s_cnt3[1] = t2; s_cnt3[2] = t3; }
+        }
+        __syncthreads();
+    };
+    uint32_t Tsel = 0;
+    for (int bit = 30; bit >= 0; bit -= 2) {
+        // candidates with the two bits set to 01, 10, 11 (ascending): keep the largest that still has k keys above it
+        const uint32_t c1 = Tsel | (1u << bit), c2 = Tsel | (2u << bit), c3 = Tsel | (3u << bit);
+        count3(c1, c2, c3);
+        if (s_cnt3[2] >= k) Tsel = c3; else if (s_cnt3[1] >= k) Tsel = c2; else if (s_cnt3[0] >= k) Tsel = c1;
+    }
+    int n_gt = 0;
+    if (Tsel != 0xffffffffu) { count3(Tsel + 1, Tsel + 1, Tsel + 1); n_gt = s_cnt3[0]; }
+    __syncthreads();
+    if (tid == 0) { s_prefix = Tsel; s_remaining = k - n_gt; }
+    __syncthreads();
     const uint32_t T = s_prefix;
     const int need_eq = s_remaining;  // elements equal to T to keep: those with the smallest indices
     if (tid == 0) { s_base_eq = 0; s_base_out = 0; }
     __syncthreads();
-    // ordered compaction, blockDim.x elements at a time
+    // ordered compaction, blockDim.x elements at a time: ranks from ballots, warp offsets from a scan by warp 0
+    __shared__ int eq_off[33], sel_off[33];
+    const int nw = blockDim.x >> 5;
     for (int start = 0; start < n; start += blockDim.x) {
         const int i = start + tid;
         const uint32_t key = i < n ? order_key(score[i]) : 0u;
         const bool gt = i < n && key > T, eq = i < n && key == T;
-        // rank of this element among the equal ones (exclusive, in index order)
-        unsigned bal = __ballot_sync(0xffffffffu, eq);
-        if (lane == 0) warp_cnt[warp] = __popc(bal);
+        const unsigned bal_eq = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) warp_cnt[warp] = __popc(bal_eq);
         __syncthreads();
-        int eq_rank = s_base_eq + __popc(bal & ((1u << lane) - 1));
-        int eq_total = 0;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { if (w < warp) eq_rank += warp_cnt[w]; eq_total += warp_cnt[w]; }
+        if (warp == 0) {
+            const int c = lane < nw ? warp_cnt[lane] : 0;
+            int inc = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += v; }
+            eq_off[lane] = inc - c;
+            if (lane == 31) eq_off[32] = inc;
+        }
+        __syncthreads();
+        const int eq_rank = s_base_eq + eq_off[warp] + __popc(bal_eq & ((1u << lane) - 1));
         const bool sel = gt || (eq && eq_rank < need_eq);
-        __syncthreads();
-        bal = __ballot_sync(0xffffffffu, sel);
+        const unsigned bal = __ballot_sync(0xffffffffu, sel);
         if (lane == 0) warp_cnt[warp] = __popc(bal);
         __syncthreads();
-        int pos = s_base_out + __popc(bal & ((1u << lane) - 1));
-        int sel_total = 0;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { if (w < warp) pos += warp_cnt[w]; sel_total += warp_cnt[w]; }
+        if (warp == 0) {
+            const int c = lane < nw ? warp_cnt[lane] : 0;
+            int inc = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += v; }
+            sel_off[lane] = inc - c;
+            if (lane == 31) sel_off[32] = inc;
+        }
+        __syncthreads();
+        const int pos = s_base_out + sel_off[warp] + __popc(bal & ((1u << lane) - 1));
         if (sel && pos < k) out[pos] = i;
         __syncthreads();
-        if (tid == 0) { s_base_eq += eq_total; s_base_out += sel_total; }
+        if (tid == 0) { s_base_eq += eq_off[32]; s_base_out += sel_off[32]; }
         __syncthreads();
     }
 }

@@ -362,6 +362,18 @@ def run_ours(args):
                 extra.append(kernel_sweep(W.CONFIGS[ci], torch, hb, HippoStep, peak))
             except Exception as e:  # noqa: BLE001
                 extra.append({"workload": W.CONFIGS[ci].name, "error": str(e)[:200]})
+        # the 64k configuration's sweep of gamma and of the pruning ratio (kept share 50/25/10/5 %)
+        base, sweep = W.CONFIGS[4], []
+        keys = ("verify_us_per_layer", "verify_frac_of_measured_peak", "draft_us_per_call", "gather_us",
+                "gather_frac_of_measured_peak", "select_us", "accept_us", "step_ms")
+        for g in W.C4_GAMMA_SWEEP:
+            for pct in W.C4_KEEP_PCT_SWEEP:
+                try:
+                    r = kernel_sweep(base.replace(gamma=g, keep_pct=pct), torch, hb, HippoStep, peak, passes=2)
+                    sweep.append({"gamma": g, "keep_pct": pct, **{k: round(r[k], 4) for k in keys}})
+                except Exception as e:  # noqa: BLE001
+                    sweep.append({"gamma": g, "keep_pct": pct, "error": str(e)[:200]})
+        extra.append({"workload": base.name + " sweep", "points": sweep})
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

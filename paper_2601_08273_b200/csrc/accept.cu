@@ -503,7 +503,6 @@ namespace hippo {
 constexpr size_t kNoAllocScratchBytes = HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_accept_scratch[kNoAllocScratchBytes];
 
-constexpr int kMaxDevices = 64;
 static void *g_scratch_addr[kMaxDevices] = {nullptr};   // device address of g_accept_scratch, per device ordinal
 static std::mutex g_scratch_mutex;
 

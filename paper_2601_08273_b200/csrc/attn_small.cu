@@ -296,10 +296,11 @@ bool attn_small_supported(const AttnParams &p, int dtype) {
 
 template <int D, int RMAX>
 static int32_t launch_small(const AttnParams &p, cudaStream_t stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    int dev;
+    if (attr_set.needed(dev)) {
         HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_small_kernel<D, RMAX>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-        attr_set = true;
+        attr_set.mark(dev);
     }
     const int pages = ceil_div(p.max_kv_len, kSmPage);
     int cs = pages < kSmMaxCluster ? pages : kSmMaxCluster;

@@ -576,6 +576,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         const int st = tid - 64;                      // 0..255
         const int quarter = warp & 3;
         const int c_first = ((warp - 2) >> 2) * 16;   // this warp's row groups: c_first, c_first + 32, ...
+        const uint32_t flip_groups = (Rp >> 4) & 1;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const int kk = quarter * 32 + lane;           // key inside the tile
         const bool d_active = (D == 128) || lane < 16;
@@ -620,6 +621,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             bool aborted = false;
             for (int i = 0; i < n; i += 2, ++it, rv.advance(n_slots), rv.advance(n_slots)) {
                 const int j = it & 1;
+                // with an odd number of 16-row groups the two warps of a quarter swap shares from tile to tile
+                const int c_tile = c_first ^ ((int)(it & flip_groups) << 4);
                 const int key0 = (tile + i) * kPageSize;
                 const int key_end = min(kvl, key0 + min(2, n - i) * kPageSize);   // first key of the tile that is not there
                 // a key that is not there compares greater than every row's limit
@@ -645,7 +648,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 // (branch-free inside; the masked variant runs only for the last tiles of a sequence)
                 float excess = -INFINITY;
                 if (!tail) {
-                    for (int c = c_first; c < Rp; c += 32) {
+                    for (int c = c_tile; c < Rp; c += 32) {
                         float sv[16];
                         tmem_ld16(s_addr + c, sv);
                         tmem_wait_ld();
@@ -657,7 +660,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                         }
                     }
                 } else {
-                    for (int c = c_first; c < Rp; c += 32) {
+                    for (int c = c_tile; c < Rp; c += 32) {
                         float sv[16];
                         tmem_ld16(s_addr + c, sv);
                         tmem_wait_ld();
@@ -675,10 +678,11 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 // a NaN excess (inf - inf on a row that has seen nothing) must count as growth
                 const bool grow = !(excess <= kRescaleThreshold);
                 const bool any_grow = softmax_bar_or(grow || !ok);
+                tc_fence_after();   // the partial sums of this tile's columns may be the other warp's stores
                 if (sh->abort) { aborted = true; break; }
                 if (any_grow) {
                     // ---- exact tile maxima per row, new references, rescale of what has been accumulated
-                    for (int c = c_first; c < Rp; c += 32) {
+                    for (int c = c_tile; c < Rp; c += 32) {
                         float sv[16];
                         tmem_ld16(s_addr + c, sv);
                         tmem_wait_ld();
@@ -717,7 +721,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                         // O^T and the partial sums hold tiles it0..it-1: wait until PV of tile it-1 has been accumulated
                         ok = W.wait(&sh->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1, 10) && ok;
                         tc_fence_after();
-                        for (int c = c_first; c < Rp; c += 32) {
+                        for (int c = c_tile; c < Rp; c += 32) {
                             float ov[16], lv[16];
                             tmem_ld16(tmem + lane_addr + col_o + c, ov);
                             tmem_ld16(tmem + lane_addr + col_l + c, lv);
@@ -735,7 +739,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 if (it >= 2) ok = W.wait(&sh->pv_done[j], ((it - 2) >> 1) & 1, 11) && ok;
                 uint8_t *pk = p_s + j * p_bytes + kk * 16;
                 const bool first_tile = it == it0;
-                for (int c = c_first; c < Rp; c += 32) {
+                for (int c = c_tile; c < Rp; c += 32) {
                     float sv[16], lv[16];
                     tmem_ld16(s_addr + c, sv);
                     if (!first_tile) tmem_ld16(tmem + lane_addr + col_l + c, lv);
@@ -769,7 +773,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             }
             if (aborted) break;
             // ---- epilogue of the segment: row sums over the keys, then O^T / l
-            for (int c = c_first; c < Rp; c += 32) {
+            // (each warp sums the columns it stored itself in the segment's last tile)
+            for (int c = c_first ^ ((int)((it - 1) & flip_groups) << 4); c < Rp; c += 32) {
                 float lv[16];
                 tmem_ld16(tmem + lane_addr + col_l + c, lv);
                 tmem_wait_ld();
@@ -1078,17 +1083,19 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     if (plan.slots < 3) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "attention: shared memory too small for %d packed rows", p.rows);
     int tmem_cols = 32;
     while (tmem_cols < 4 * Rp) tmem_cols *= 2;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    int dev;
+    if (attr_set.needed(dev)) {
         HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         HIPPO_CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-        attr_set = true;
+        attr_set.mark(dev);
     }
     const int units = p.batch * p.n_kv_heads;
-    // resident clusters per cluster size, asked once per ring size (the only launch parameter that moves it)
+    // resident clusters per cluster size, asked once per ring size (the only launch parameter that moves it); every
+    // device of this library's only target has the same answer, so one table serves them all
     static int max_active[kMaxSlots + 1][17];
-    static bool have_active[kMaxSlots + 1] = {false};
-    if (!have_active[plan.slots]) {
+    static std::atomic<bool> have_active[kMaxSlots + 1];
+    if (!have_active[plan.slots].load(std::memory_order_acquire)) {
         for (int c = 2; c <= 16; ++c) {
             cudaLaunchConfig_t q = {};
             cudaLaunchAttribute qa[1];
@@ -1100,7 +1107,7 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
             if (cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<D>, &q) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
             max_active[plan.slots][c] = n;
         }
-        have_active[plan.slots] = true;
+        have_active[plan.slots].store(true, std::memory_order_release);
     }
     const int cs = p.num_splits > 0 ? 0 : choose_cluster_size(units, ceil_div(p.max_kv_len, kBlockN), max_active[plan.slots]);
     // Both kernels are launched with programmatic stream serialization and wait (griddepcontrol.wait) before they

@@ -3,6 +3,7 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <atomic>
 #include <stdint.h>
 #include <stdio.h>
 
@@ -35,6 +36,19 @@ int32_t cuda_fail(cudaError_t e, const char *what);
         cudaError_t e_ = (expr);                               \
         if (e_ != cudaSuccess) return ::hippo::cuda_fail(e_, #expr); \
     } while (0)
+
+// Function attributes and occupancy answers belong to a device: one flag per device ordinal, set after the first
+// successful set-up there.  Two threads racing on a device's first call both do the set-up, which is harmless.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    std::atomic<bool> done[kMaxDevices];
+    // true when the current device still needs its set-up; dev receives the ordinal (-1: unknown, always set up)
+    bool needed(int &dev) {
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { dev = -1; return true; }
+        return !done[dev].load(std::memory_order_acquire);
+    }
+    void mark(int dev) { if (dev >= 0) done[dev].store(true, std::memory_order_release); }
+};
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

@@ -518,13 +518,14 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
     }
     if (score_mask & HIPPO_SCORE_SPA) {
         dim3 g2((unsigned)(frames * p.crops_y * p.crops_x));
-        static bool spa_attr = false;
-        if (!spa_attr) {
+        static PerDeviceOnce spa_attr;
+        int dev;
+        if (spa_attr.needed(dev)) {
             HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<float, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<5>::kSmemBytes));
             HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<__nv_bfloat16, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<5>::kSmemBytes));
             HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<float, 7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<7>::kSmemBytes));
             HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<__nv_bfloat16, 7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<7>::kSmemBytes));
-            spa_attr = true;
+            spa_attr.mark(dev);
         }
         if (crop_h * crop_w <= 25) {
             if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float, 5><<<g2, SpaShape<5>::kThreads, SpaShape<5>::kSmemBytes, s>>>(p);

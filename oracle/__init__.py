@@ -136,6 +136,24 @@ def attention(q, k, v, kv_len: Sequence[int], scale: Optional[float] = None, row
     return out, lse
 
 
+def attention_mass(q_txt, k_vid, n_visual: Sequence[int], scale: Optional[float] = None) -> np.ndarray:
+    """Eq. 2: mean over layers, heads and text rows of softmax_j(scale q_i . k_j) over the visual keys.
+
+    q_txt [n_layers][B][L_txt][H_q][D]; k_vid [n_layers][B][max_nv][H_kv][D].  Returns float64 [B][max_nv]
+    (zeros at and beyond n_visual[b]).
+    """
+    q, k = _f32(q_txt), _f32(k_vid)
+    nl, B, L_txt, Hq, D = q.shape
+    _, _, max_nv, Hkv, _ = k.shape
+    nv = _i32(n_visual)
+    sc = ctypes.c_double(1.0 / np.sqrt(D) if scale is None else scale)
+    mass = np.empty((B, max_nv), dtype=np.float64)
+    rc = _load().oracle_attention_mass(nl, B, L_txt, Hq, Hkv, D, max_nv, _p(nv), _p(q), _p(k), sc, _p(mass))
+    if rc != 0:
+        raise ValueError("oracle_attention_mass rc=%d" % rc)
+    return mass
+
+
 def accept(target_logits, draft_logits, draft_tokens, u_accept, u_resample):
     """Eq. 1 + residual resample / bonus.  Returns (n_accepted [B], out_tokens [B][gamma+1],
     margin_accept [B], margin_cdf [B])."""

@@ -17,6 +17,7 @@
  *                       paper, so parity with the authors' own code is unpinned.
  *   top-k, gather     - pinned (library sort / exact copy identities).
  *   attention         - pinned (library softmax-attention, closed forms).
+ *   attention mass    - pinned (hand-worked case, closed forms, library softmax, invariants).
  *   acceptance        - pinned (losslessness identity by enumeration and by seeded simulation).
  */
 #include <math.h>
@@ -294,6 +295,56 @@ int oracle_attention_rows(int n_sel, const int32_t *sel_b, const int32_t *sel_t,
     for (int r = 0; r < n_sel; ++r)
         attention_row(sel_b[r], sel_t[r], sel_h[r], q_len, Hq, Hkv, D, max_kv, kv_len[sel_b[r]], q, k, v, scale,
                       out + (size_t)r * D, lse ? lse + r : NULL);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Global semantic relevance (Section 5.1, Eq. 2).  For every layer l, attention head h and text query
+ * row i the cross-modal attention row is S_i = softmax over the N_v visual keys of scale * q_i . k_j
+ * (head h reads KV head h / (H_q / H_kv)); the score of visual token j is the mean of [S]_ij over
+ * layers, heads and text rows.  The softmax runs over the visual keys only: S_attn is defined as an
+ * L_txt x N_v matrix.
+ * q_txt [n_layers][B][L_txt][H_q][D]; k_vid [n_layers][B][max_nv][H_kv][D]; n_visual [B];
+ * mass double [B][max_nv] (entries at and beyond n_visual[b] are set to 0).
+ * ---------------------------------------------------------------------------------------------- */
+int oracle_attention_mass(int n_layers, int B, int L_txt, int Hq, int Hkv, int D, int max_nv, const int32_t *n_visual,
+                          const float *q_txt, const float *k_vid, double scale, double *mass) {
+    if (n_layers <= 0 || B <= 0 || L_txt <= 0 || Hkv <= 0 || Hq % Hkv || D <= 0 || max_nv <= 0) return -1;
+    int G = Hq / Hkv;
+    double *head_sum = (double *)malloc((size_t)Hq * max_nv * sizeof(double));   /* sum over text rows, one head */
+    if (!head_sum) return -2;
+    for (size_t x = 0; x < (size_t)B * max_nv; ++x) mass[x] = 0.0;
+    for (int b = 0; b < B; ++b) {
+        int nv = n_visual[b];
+        if (nv <= 0) continue;
+        if (nv > max_nv) { free(head_sum); return -1; }
+        for (int l = 0; l < n_layers; ++l) {
+            const float *ql = q_txt + ((size_t)l * B + b) * L_txt * Hq * D;
+            const float *kl = k_vid + ((size_t)l * B + b) * max_nv * Hkv * D;
+#pragma omp parallel for schedule(dynamic, 1)
+            for (int h = 0; h < Hq; ++h) {
+                int hk = h / G;
+                double *acc = head_sum + (size_t)h * max_nv;
+                double *a = (double *)malloc((size_t)nv * sizeof(double));
+                for (int j = 0; j < nv; ++j) acc[j] = 0.0;
+                for (int i = 0; i < L_txt; ++i) {
+                    const float *qr = ql + ((size_t)i * Hq + h) * D;
+                    double m = -INFINITY, z = 0.0;
+                    for (int j = 0; j < nv; ++j) {
+                        a[j] = scale * dot_ff(qr, kl + ((size_t)j * Hkv + hk) * D, D);
+                        if (a[j] > m) m = a[j];
+                    }
+                    for (int j = 0; j < nv; ++j) { a[j] = exp(a[j] - m); z += a[j]; }
+                    for (int j = 0; j < nv; ++j) acc[j] += a[j] / z;
+                }
+                free(a);
+            }
+            for (int h = 0; h < Hq; ++h)
+                for (int j = 0; j < nv; ++j) mass[(size_t)b * max_nv + j] += head_sum[(size_t)h * max_nv + j];
+        }
+        for (int j = 0; j < nv; ++j) mass[(size_t)b * max_nv + j] /= (double)n_layers * Hq * L_txt;
+    }
+    free(head_sum);
     return 0;
 }
 

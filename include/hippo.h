@@ -7,6 +7,7 @@
  *   hippo_draft_attention   draft decode attention over the pruned KV (Section 3.2, drafting phase)
  *   hippo_verify_attention  target verification attention, gamma+1 query tokens (Section 3.2)
  *   hippo_accept            lossless speculative acceptance (Section 3.2, Eq. 1 and the resampling rule)
+ * and, upstream of the selection, hippo_attention_mass (global semantic relevance, Section 5.1, Eq. 2).
  *
  * Conventions
  *   - Every call returns a hippo_status_t (0 = HIPPO_OK, negative = error).  Arguments are validated on the
@@ -91,6 +92,28 @@ int32_t hippo_workspace_status(const void *workspace, void *stream);
 /* Zeroes the header of a workspace (status word and arrival counters); enqueued on `stream`.  Must be called
  * once on a fresh workspace before its first use by the attention calls, and after a reported time-out. */
 int32_t hippo_workspace_reset(void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- global semantic relevance: Section 5.1, Eq. 2 ------------------------------------------------------------ */
+/*
+ * The attention mass that hippo_select_tokens takes as `attn_mass`, from the prefilled target cache: for every
+ * text query row i and attention head h, S_i = softmax over the VISUAL keys j < n_visual[b] of
+ * scale * q_txt[b][i][h] . K[b][j][h / G]; Eq. 2 is the mean of [S_i]_j over layers, heads and text rows.
+ * One call handles one layer and ADDS its share:
+ *     mass[off_b + j] += weight * sum_{h, i} [S_i^(h)]_j        off_b = sum(n_visual[0..b))
+ * so zeroing `mass` and calling once per layer with weight = 1 / (n_layers * n_q_heads * l_txt) yields Eq. 2.
+ * The visual tokens are positions [0, n_visual[b]) of sequence b in the cache (text and generated tokens follow);
+ * only the key pool is read.
+ *   n_visual  host int32 [batch], each >= 0; batch <= 64      q_txt  [batch][l_txt][n_q_heads][head_dim], kv dtype
+ *   softmax_scale  0 selects 1/sqrt(head_dim)                  mass   fp32 [sum n_visual], read and written
+ * bf16 with head_dim 64 or 128 and l_txt * G <= 3072 runs on the tensor cores (logits formed twice, never stored);
+ * other shapes and fp32 run on the CUDA cores.  Sums are added in a fixed order: results are reproducible.
+ * The workspace needs no reset for this call unless a time-out was reported.
+ */
+size_t hippo_attention_mass_workspace_bytes(int32_t batch, const int32_t *n_visual, int32_t l_txt, int32_t n_q_heads,
+                                            int32_t n_kv_heads, int32_t head_dim, int32_t dtype);
+int32_t hippo_attention_mass(int32_t batch, const int32_t *n_visual, int32_t l_txt, int32_t n_q_heads,
+                             const void *q_txt, const hippo_kv_cache_t *kv, float softmax_scale, float weight,
+                             float *mass, void *workspace, size_t workspace_bytes, void *stream);
 
 /* ---- selection: Section 5.1 --------------------------------------------------------------------------------- */
 /*

@@ -70,6 +70,10 @@ lib.hippo_attention_workspace_bytes.argtypes = [_i32] * 5
 for _name in ("hippo_verify_attention", "hippo_draft_attention"):
     getattr(lib, _name).restype = _i32
     getattr(lib, _name).argtypes = [_i32, _i32, _i32, _vp, _KVP, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _sz, _vp]
+lib.hippo_attention_mass_workspace_bytes.restype = _sz
+lib.hippo_attention_mass_workspace_bytes.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32, _i32]
+lib.hippo_attention_mass.restype = _i32
+lib.hippo_attention_mass.argtypes = [_i32, _I32P, _i32, _i32, _vp, _KVP, _f32, _f32, _vp, _vp, _sz, _vp]
 lib.hippo_accept_workspace_bytes.restype = _sz
 lib.hippo_accept_workspace_bytes.argtypes = [_i32, _i32, _i32]
 lib.hippo_accept.restype = _i32
@@ -232,6 +236,30 @@ def hippo_draft_attention(q: torch.Tensor, kv: KVCache, kv_len: torch.Tensor, ma
                           lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
     return _attention(lib.hippo_draft_attention, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse,
                       workspace, stream)
+
+
+# ---- global semantic relevance (Eq. 2) ----------------------------------------------------------------------------
+
+def hippo_attention_mass_workspace_bytes(n_visual: Sequence[int], l_txt: int, n_q_heads: int, n_kv_heads: int,
+                                         head_dim: int, dtype: int) -> int:
+    return int(lib.hippo_attention_mass_workspace_bytes(len(n_visual), _host_i32(n_visual), l_txt, n_q_heads,
+                                                        n_kv_heads, head_dim, dtype))
+
+
+def hippo_attention_mass(q_txt: torch.Tensor, kv: "KVCache", n_visual: Sequence[int], weight: float,
+                         mass: torch.Tensor, softmax_scale: float = 0.0, workspace: Optional[torch.Tensor] = None,
+                         stream=None) -> torch.Tensor:
+    """One layer's share of Eq. 2, added into `mass` (fp32 [sum n_visual]).  q_txt [B][l_txt][H_q][D]."""
+    B, l_txt, hq, D = q_txt.shape
+    assert q_txt.is_contiguous() and mass.dtype == torch.float32 and mass.is_contiguous()
+    assert len(n_visual) == B and mass.numel() >= sum(int(x) for x in n_visual)
+    if workspace is None:
+        workspace = new_workspace(hippo_attention_mass_workspace_bytes(n_visual, l_txt, hq, kv.struct.n_kv_heads,
+                                                                        D, _dtype_code(q_txt)), q_txt.device)
+    _check(lib.hippo_attention_mass(B, _host_i32(n_visual), l_txt, hq, _ptr(q_txt), ctypes.byref(kv.struct),
+                                    float(softmax_scale), float(weight), _ptr(mass), _ptr(workspace),
+                                    workspace.numel(), _stream(stream)))
+    return mass
 
 
 # ---- acceptance ---------------------------------------------------------------------------------------------------

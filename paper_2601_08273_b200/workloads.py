@@ -81,7 +81,7 @@ def rng_for(cfg: HippoConfig, tag: int, sub: int = 0) -> np.random.Generator:
     return np.random.default_rng([cfg.seed, tag, sub])
 
 
-TAG_LEN, TAG_EMB, TAG_MASS, TAG_ATT_T, TAG_ATT_D, TAG_ACC, TAG_PAGES, TAG_GATHER = range(8)
+TAG_LEN, TAG_EMB, TAG_MASS, TAG_ATT_T, TAG_ATT_D, TAG_ACC, TAG_PAGES, TAG_GATHER, TAG_QTXT = range(9)
 
 # ------------------------------------------------------------------------------------------------
 # storage rounding
@@ -173,6 +173,29 @@ def select_inputs(cfg: HippoConfig, b: int = 0, n_visual: Optional[int] = None) 
     emb = round_to_storage(normal_f32(r, (n_v, cfg.embed_dim)), cfg.dtype)
     return {"n_visual": n_v, "embeds": emb, "attn_mass": attention_mass(cfg, n_v, b),
             "k": keep_count(n_v, cfg.keep_pct)}
+
+def mass_inputs(cfg: HippoConfig, n_visual: List[int], layer: int = 0) -> Dict[str, np.ndarray]:
+    """Text queries and visual keys of one target layer for the global-relevance score.
+
+    q_txt [B][n_text][H_q][D], k_vid [B][max(n_visual)][H_kv][D].  Both are N(0,1) plus a component along one shared
+    direction sized so that the resulting text-to-visual attention follows the configuration's mass profile
+    (power law with inflated frame borders) up to the random part of the logits."""
+    hq, hkv, d = cfg.tgt_q_heads, cfg.tgt_kv_heads, cfg.tgt_head_dim
+    r = rng_for(cfg, TAG_QTXT, layer)
+    B, T = len(n_visual), max(max(n_visual), 1)
+    u = r.standard_normal(d)
+    u = (u / np.linalg.norm(u)).astype(np.float32)
+    q = normal_f32(r, (B, cfg.n_text, hq, d)) + np.float32(4.0) * u
+    k = normal_f32(r, (B, T, hkv, d))
+    scale = 1.0 / np.sqrt(d)
+    for b, nv in enumerate(n_visual):
+        if nv <= 0:
+            continue
+        w = attention_mass(cfg, nv, b).astype(np.float64)
+        bias = np.log(w / w.max()) / (4.0 * scale)
+        k[b, :nv] += (bias[:, None, None] * u[None, None, :]).astype(np.float32)
+    return {"q_txt": round_to_storage(q, cfg.dtype), "k_vid": round_to_storage(k, cfg.dtype)}
+
 
 # ------------------------------------------------------------------------------------------------
 # attention inputs (logical layout [B][T][H_kv][D]) and the paged pool layout

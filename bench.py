@@ -226,6 +226,12 @@ def kernel_sweep(cfg, torch, hb, HippoStep, peak, passes=3, max_gb=24.0):
     out.update({"draft_us_per_call": dms * 1e3, "draft_kv_mb_per_call": st.draft_kv_bytes_per_call(cfg.gamma // 2) / 1e6})
     st.accept(cur)
     out["accept_us"] = timed(lambda: st.accept(cur), 10, cur, torch) / 10 * 1e3
+    # global semantic relevance (Eq. 2) over the timed target layers: bound by the exponentials (MUFU: 16 / clk / SM)
+    st.attention_mass(cur)
+    mms = timed(lambda: st.attention_mass(cur), 2, cur, torch) / (2 * layers)
+    mufu_peak = 148 * 16 * 1.965e9
+    out.update({"mass_us_per_layer": mms * 1e3, "mass_gexp_per_s": st.mass_exps_per_layer() / mms / 1e6,
+                "mass_frac_of_mufu_peak": st.mass_exps_per_layer() / (mms * 1e-3) / mufu_peak})
     # the whole step: select -> gather -> (draft || verify on two streams) -> accept, all target layers if they fit
     st.run()
     torch.cuda.synchronize()
@@ -349,6 +355,9 @@ def run_ours(args):
             fn()
             breakdown[name + "_us"] = timed(fn, reps, cur, torch) / reps * 1e3
         breakdown["verify_all_us"] = verify_ms / steps * 1e3
+        st.attention_mass(cur)
+        breakdown["mass_all_layers_us"] = timed(lambda: st.attention_mass(cur), 3, cur, torch) / 3 * 1e3
+        breakdown["mass_gexp_per_s"] = st.mass_exps_per_layer() * st.Lt / breakdown["mass_all_layers_us"] / 1e3
         breakdown["draft_us_per_call"] = breakdown["draft_all_us"] / (cfg.gamma * st.Ld)
         breakdown["gather_gbps"] = st.gather_bytes() / breakdown["gather_us"] / 1e3
         breakdown["draft_gbps"] = st.draft_kv_bytes_per_call(cfg.gamma // 2) / breakdown["draft_us_per_call"] / 1e3

@@ -18,7 +18,8 @@
 // block takes T = floor(128 / G) text rows, fetched with one 4-D TMA box per 64 columns straight into the
 // 128-byte-swizzled operand layout.  Keys come in 128-key tiles = two 64-token pages, as in the attention kernels.
 //
-// CTA = 6 warps: warp 0 TMA producer, warp 1 MMA issuer and tensor-memory owner, warps 2-5 consumers.
+// CTA = 18 warps: warp 0 TMA producer, warp 1 MMA issuer and tensor-memory owner, warps 2-17 consumers (a warp reads
+// its quarter of the tensor-memory lanes and one 32-column slice of the tile).
 // The work is bound by the exponentials (one per row and key in each pass), not by the MMAs or by memory.
 // Every mbarrier wait is bounded; on expiry the CTA records HIPPO_ERR_TIMEOUT in the workspace header and exits.
 //
@@ -31,11 +32,14 @@
 
 namespace hippo {
 
-constexpr int kMassThreads = 192;
-constexpr int kMassConsumers = 128;
+constexpr int kMassSlices = 4;            // column slices of an accumulator tile, one consumer warp each per lane quarter
+constexpr int kMassSliceCols = 32;
+constexpr int kMassConsumers = 128 * kMassSlices;
+constexpr int kMassThreads = 64 + kMassConsumers;
 constexpr int kMassSlots = 3;            // ring of streamed tiles
 constexpr int kMassTile = 128;           // rows and keys per accumulator tile
 constexpr int kMassMaxBatch = 64;        // per-sequence lengths travel in the kernel parameters
+constexpr int kMassMaxSplits = 64;
 constexpr int kMassMaxRows = 3072;       // l_txt * group: the pass-2 table of a KV head lives in shared memory
 constexpr float kMassLog2e = 1.4426950408889634f;
 constexpr unsigned long long kMassWaitLimitNs = 2000000000ull;
@@ -106,7 +110,8 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
     uint8_t *ring = res + 2 * kTileBytes;                 // [kMassSlots] streamed tiles, same layout
     float2 *tab = (float2 *)(ring + kMassSlots * kTileBytes);   // pass 1 only: (-max, 1 / sum) of the KV head's rows
     const int tab_entries = PASS == 1 ? ((p.r_tot + 16 + 15) & ~15) : 0;
-    MassShared *sh = (MassShared *)(tab + tab_entries);
+    float2 *part = tab + tab_entries;                       // [2][kMassSlices][128]: the slices' partial results
+    MassShared *sh = (MassShared *)(part + 2 * kMassSlices * kMassTile);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.group, Hkv = p.n_kv_heads, T = p.t_per_block, TG = p.rows_per_block;
@@ -243,98 +248,128 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
             mass_wait(sh, hdr, &sh->drain, 0, 8);
         }
     } else {
-        // ================= consumers: thread = one tensor-memory lane = one row of the accumulator tile ========
-        const int quarter = warp & 3;
+        // ================= consumers =================
+        // A thread owns one tensor-memory lane (a row of the accumulator tile) and one 32-column slice of it; the four
+        // slices of a lane run on four warps of the same scheduler, which hides the tensor-memory and MUFU latencies.
+        // Control flow is the same for all consumer warps whatever `ok` is: they meet at one named barrier per outer step.
+        const int quarter = warp & 3, slice = (warp - 2) >> 2;
         const int L = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const float sl2 = p.sl2;
+        const int c0 = slice * kMassSliceCols;
         uint32_t it = 0;
         bool ok = true;
-        for (int o = o0; o < o1 && ok; ++o) {
+        for (int o = o0; o < o1; ++o) {
             float m = -INFINITY, l = 0.f, acc = 0.f;
             for (int i = i0; i < i1; ++i, ++it) {
                 const int j = it & 1;
-                ok = mass_wait(sh, hdr, &sh->s_full[j], (it >> 1) & 1, 9);
-                if (!ok) break;
+                if (ok) ok = mass_wait(sh, hdr, &sh->s_full[j], (it >> 1) & 1, 9);
+                if (!ok) continue;
                 tc_fence_after();
-                const uint32_t s_addr = tmem + lane_addr + j * kMassTile;
-                if (PASS == 0) {
-                    // columns = keys of tile i
-                    const int ncols = min(kMassTile, nv - i * kMassTile);
-                    float tmax = -INFINITY;
-                    for (int c = 0; c < ncols; c += 16) {
-                        float sv[16];
-                        tmem_ld16(s_addr + c, sv);
-                        tmem_wait_ld();
-                        if (c + 16 <= ncols) {
+                // columns: keys of tile i (pass 0) / packed rows of block i (pass 1)
+                const int ncols = PASS == 0 ? min(kMassTile, nv - i * kMassTile) : min(TG, p.r_tot - i * TG);
+                const int mine = min(kMassSliceCols, ncols - c0);      // valid columns of this slice
+                if (mine > 0) {
+                    float sv[kMassSliceCols];
+                    const uint32_t s_addr = tmem + lane_addr + j * kMassTile + c0;
+                    tmem_ld16(s_addr, sv);
+                    tmem_ld16(s_addr + 16, sv + 16);
+                    tmem_wait_ld();
+                    if (PASS == 0) {
+                        float tmax = -INFINITY;
+                        if (mine == kMassSliceCols) {
+                            float t4[4] = {sv[0], sv[1], sv[2], sv[3]};     // four short chains instead of one long one
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) tmax = fmaxf(tmax, sv[e]);
+                            for (int e = 4; e < kMassSliceCols; ++e) t4[e & 3] = fmaxf(t4[e & 3], sv[e]);
+                            tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) tmax = fmaxf(tmax, c + e < ncols ? sv[e] : -INFINITY);
+                            for (int e = 0; e < kMassSliceCols; ++e) tmax = fmaxf(tmax, e < mine ? sv[e] : -INFINITY);
                         }
-                    }
-                    const float m_new = fmaxf(m, tmax * sl2);
-                    l *= ex2_approx(m - m_new);     // m = -inf on the first tile: factor 0
-                    m = m_new;
-                    const float mneg = -m_new;
-                    float add0 = 0.f, add1 = 0.f;
-                    for (int c = 0; c < ncols; c += 16) {
-                        float sv[16];
-                        tmem_ld16(s_addr + c, sv);
-                        tmem_wait_ld();
-                        if (c + 16 <= ncols) {
+                        const float m_new = fmaxf(m, tmax * sl2);
+                        l *= ex2_approx(m - m_new);     // m = -inf at first: factor 0
+                        m = m_new;
+                        const float mneg = -m_new;
+                        float add0 = 0.f, add1 = 0.f;
+                        if (mine == kMassSliceCols) {
+                            float add2 = 0.f, add3 = 0.f;
 #pragma unroll
-                            for (int e = 0; e < 16; e += 2) {
+                            for (int e = 0; e < kMassSliceCols; e += 4) {
                                 add0 += ex2_approx(fmaf(sv[e], sl2, mneg));
                                 add1 += ex2_approx(fmaf(sv[e + 1], sl2, mneg));
+                                add2 += ex2_approx(fmaf(sv[e + 2], sl2, mneg));
+                                add3 += ex2_approx(fmaf(sv[e + 3], sl2, mneg));
                             }
+                            add0 += add2; add1 += add3;
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) {
+                            for (int e = 0; e < kMassSliceCols; ++e) {
                                 const float pe = ex2_approx(fmaf(sv[e], sl2, mneg));
-                                add0 += c + e < ncols ? pe : 0.f;
+                                add0 += e < mine ? pe : 0.f;
                             }
                         }
-                    }
-                    l += add0 + add1;
-                } else {
-                    // columns = packed rows of block i
-                    const int ncols = min(TG, p.r_tot - i * TG);
-                    const float2 *tb = tab + i * TG;
-                    float a0 = 0.f, a1 = 0.f;
-                    for (int c = 0; c < ncols; c += 16) {
-                        float sv[16];
-                        tmem_ld16(s_addr + c, sv);
-                        tmem_wait_ld();
-                        if (c + 16 <= ncols) {
+                        l += add0 + add1;
+                    } else {
+                        const float2 *tb = tab + i * TG + c0;
+                        float a0 = 0.f, a1 = 0.f;
+                        if (mine == kMassSliceCols && ((i * TG) & 1) == 0) {
+                            // two table entries per 16-byte load (the block's first entry is 16-byte aligned)
+                            float a2 = 0.f, a3 = 0.f;
+                            const float4 *tb4 = reinterpret_cast<const float4 *>(tb);
 #pragma unroll
-                            for (int e = 0; e < 16; e += 2) {
-                                const float2 t0 = tb[c + e], t1 = tb[c + e + 1];
+                            for (int e = 0; e < kMassSliceCols; e += 4) {
+                                const float4 t0 = tb4[e >> 1], t1 = tb4[(e >> 1) + 1];
+                                a0 = fmaf(ex2_approx(fmaf(sv[e], sl2, t0.x)), t0.y, a0);
+                                a1 = fmaf(ex2_approx(fmaf(sv[e + 1], sl2, t0.z)), t0.w, a1);
+                                a2 = fmaf(ex2_approx(fmaf(sv[e + 2], sl2, t1.x)), t1.y, a2);
+                                a3 = fmaf(ex2_approx(fmaf(sv[e + 3], sl2, t1.z)), t1.w, a3);
+                            }
+                            a0 += a2; a1 += a3;
+                        } else if (mine == kMassSliceCols) {
+#pragma unroll
+                            for (int e = 0; e < kMassSliceCols; e += 2) {
+                                const float2 t0 = tb[e], t1 = tb[e + 1];
                                 a0 = fmaf(ex2_approx(fmaf(sv[e], sl2, t0.x)), t0.y, a0);
                                 a1 = fmaf(ex2_approx(fmaf(sv[e + 1], sl2, t1.x)), t1.y, a1);
                             }
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) {
-                                const float2 t0 = tb[c + e];
+                            for (int e = 0; e < kMassSliceCols; ++e) {
+                                const float2 t0 = tb[e];
                                 const float pe = ex2_approx(fmaf(sv[e], sl2, t0.x)) * t0.y;
-                                a0 += c + e < ncols ? pe : 0.f;
+                                a0 += e < mine ? pe : 0.f;
                             }
                         }
+                        acc += a0 + a1;
                     }
-                    acc += a0 + a1;
                 }
                 tc_fence_before();
                 mbar_arrive(smem_u32(&sh->s_free[j]));
             }
-            if (!ok) break;
-            if (PASS == 0) {
-                if (L < TG && o * TG + L < p.r_tot)
-                    p.stats[((size_t)unit * p.stat_splits + split) * p.r_tot + o * TG + L] = make_float2(m, l);
-            } else {
-                const int key = o * kMassTile + L;
-                if (key < nv) p.colsum[(size_t)hk * p.sum_nv + p.offset[b] + key] = acc;
+            // the four slices of a lane meet in shared memory (double buffered over the outer steps)
+            float2 *pt = part + ((o - o0) & 1) * (kMassSlices * kMassTile);
+            pt[slice * kMassTile + L] = PASS == 0 ? make_float2(m, l) : make_float2(acc, 0.f);
+            asm volatile("bar.sync 1, %0;" ::"n"(kMassConsumers) : "memory");
+            if (slice == 0 && ok && !sh->abort) {
+                if (PASS == 0) {
+                    float M = m;
+#pragma unroll
+                    for (int q = 1; q < kMassSlices; ++q) M = fmaxf(M, pt[q * kMassTile + L].x);
+                    float Ls = 0.f;
+#pragma unroll
+                    for (int q = 0; q < kMassSlices; ++q) {
+                        const float2 v = pt[q * kMassTile + L];
+                        if (v.y > 0.f) Ls += v.y * ex2_approx(v.x - M);
+                    }
+                    if (L < TG && o * TG + L < p.r_tot)
+                        p.stats[((size_t)unit * p.stat_splits + split) * p.r_tot + o * TG + L] = make_float2(M, Ls);
+                } else {
+                    float sum = acc;
+#pragma unroll
+                    for (int q = 1; q < kMassSlices; ++q) sum += pt[q * kMassTile + L].x;
+                    const int key = o * kMassTile + L;
+                    if (key < nv) p.colsum[(size_t)hk * p.sum_nv + p.offset[b] + key] = sum;
+                }
             }
         }
     }
@@ -432,6 +467,19 @@ struct MassPlan {
     size_t stats_off, table_off, colsum_off, total;
 };
 
+// Key splits for `items` equal work items of `tiles` key tiles each (every key tile costing `inner` accumulator
+// tiles): the CTAs run one per SM in waves, so the cost is waves x (accumulator tiles per CTA + a fixed start-up).
+static int mass_best_splits(int items, int tiles, int inner) {
+    int best = 1;
+    long long best_cost = -1;
+    for (int s = 1; s <= tiles && s <= kMassMaxSplits; ++s) {
+        const long long waves = ((long long)items * s + kNumSMs - 1) / kNumSMs;
+        const long long cost = waves * ((long long)ceil_div(tiles, s) * inner + 4);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    return best;
+}
+
 static MassPlan mass_plan(int batch, const int32_t *n_visual, int l_txt, int n_q_heads, int n_kv_heads, int head_dim, int dtype) {
     MassPlan pl;
     const int G = n_q_heads / n_kv_heads;
@@ -446,10 +494,8 @@ static MassPlan mass_plan(int batch, const int32_t *n_visual, int l_txt, int n_q
     for (int b = 0; b < batch; ++b) { sum_nv += n_visual[b]; if (n_visual[b] > max_nv) max_nv = n_visual[b]; }
     pl.max_nkt = ceil_div(max_nv > 0 ? max_nv : 1, kMassTile);
     const int units = batch * n_kv_heads;
-    pl.stat_splits = pl.tc ? ceil_div(2 * kNumSMs, units * pl.RB) : 1;
-    if (pl.stat_splits > pl.max_nkt) pl.stat_splits = pl.max_nkt;
-    pl.sum_splits = ceil_div(2 * kNumSMs, units);
-    if (pl.sum_splits > pl.max_nkt) pl.sum_splits = pl.max_nkt;
+    pl.stat_splits = pl.tc ? mass_best_splits(units * pl.RB, pl.max_nkt, 1) : 1;
+    pl.sum_splits = mass_best_splits(units, pl.max_nkt, pl.RB);
     pl.stats_off = kWsHeaderBytes;
     pl.table_off = align_up(pl.stats_off + (size_t)units * pl.stat_splits * pl.r_tot * sizeof(float2), 256);
     pl.colsum_off = align_up(pl.table_off + (size_t)units * pl.r_tot * sizeof(float2), 256);
@@ -493,7 +539,7 @@ static int32_t launch_mass_tc(MassParams &p, const MassPlan &pl, long long pool_
     rc = make_q_map(&qm, p.q, p.batch, p.l_txt, p.n_q_heads, D, p.group, pl.T);
     if (rc != HIPPO_OK) return rc;
     const size_t tiles = (size_t)(2 + kMassSlots) * kMassTile * D * 2;
-    const size_t smem0 = 1024 + tiles + sizeof(MassShared) + 64;
+    const size_t smem0 = 1024 + tiles + 2 * kMassSlices * kMassTile * sizeof(float2) + sizeof(MassShared) + 64;
     const size_t smem1 = smem0 + (size_t)((p.r_tot + 16 + 15) & ~15) * sizeof(float2);
     static PerDeviceOnce attr_set;
     int dev;

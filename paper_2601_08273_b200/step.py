@@ -156,6 +156,31 @@ class HippoStep:
             hb.hippo_verify_attention(self.q_t[l], self.tgt_cache[l], self.kv_len_t, m, out=self.out_t[l],
                                       workspace=self.verify_ws, stream=stream)
 
+    def attention_mass(self, stream=None):
+        """Eq. 2 over all target layers of the prefilled cache (once per prompt, upstream of select); the result goes
+        to `self.mass_out`, the step's own selection keeps reading the configuration's synthetic mass."""
+        c = self.cfg
+        if getattr(self, "q_txt", None) is None:
+            gen = torch.Generator(device=self.device)
+            gen.manual_seed(2000 + c.seed)
+            self.q_txt = _randn((self.Lt, c.batch, c.n_text, c.tgt_q_heads, c.tgt_head_dim), self.tdt, gen, self.device)
+            self.mass_out = torch.zeros(sum(self.n_visual), dtype=torch.float32, device=self.device)
+            code = hb.HIPPO_DTYPE_FP32 if c.dtype == "fp32" else hb.HIPPO_DTYPE_BF16
+            self.mass_ws = hb.new_workspace(hb.hippo_attention_mass_workspace_bytes(
+                self.n_visual, c.n_text, c.tgt_q_heads, c.tgt_kv_heads, c.tgt_head_dim, code), self.device)
+        w = 1.0 / (self.Lt * c.tgt_q_heads * c.n_text)
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        with torch.cuda.stream(s):
+            self.mass_out.zero_()
+        for l in range(self.Lt):
+            hb.hippo_attention_mass(self.q_txt[l], self.tgt_cache[l], self.n_visual, w, self.mass_out,
+                                    workspace=self.mass_ws, stream=stream)
+
+    def mass_exps_per_layer(self) -> int:
+        """Exponentials Eq. 2 needs per layer as computed here: one per (text row, head, visual key) in each pass."""
+        c = self.cfg
+        return 2 * c.n_text * c.tgt_q_heads * sum(self.n_visual)
+
     def accept(self, stream=None):
         a = self.acc
         hb.hippo_accept(a["target_logits"], a["draft_logits"], a["draft_tokens"], a["u_accept"], a["u_resample"],

@@ -7,9 +7,9 @@
 // times on the tensor cores (bf16, head_dim 64 or 128), and never stored:
 //   pass 1 (row statistics)  S   [128 rows x 128 keys] = Q_block . K_tile^T    thread = row: running max and sum of
 //                                                                                exponentials over its CTA's key tiles
-//   merge                     the key splits of a row -> (-max, 1 / sum)
+//   merge                     the key splits of a row -> t = -(max + log2 sum)
 //   pass 2 (column sums)      S^T [128 keys x 128 rows] = K_tile . Q_block^T    thread = key: sum over the rows of
-//                                                                                2^(s - max_row) / sum_row
+//                                                                                2^(s + t_row)
 //   reduce                    mass += weight * (sum of the KV heads' column sums), in a fixed order
 // Both passes are one kernel: a "resident" tile is the A operand (the Q block in pass 1, the key tile in pass 2) and
 // the other operand streams through a ring of shared-memory slots; the accumulator tile lives in tensor memory,
@@ -61,7 +61,8 @@ struct MassParams {
     const void *q;
     const void *k_pages;
     float2 *stats;         // [batch * n_kv_heads][stat_splits][r_tot]: (max in the log2 domain, sum of 2^(x - max))
-    float2 *table;         // [batch * n_kv_heads][r_tot]: (-max, 1 / sum)
+    float2 *table;         // CUDA-core path: [batch * n_kv_heads][r_tot] (-max, 1 / sum), natural-log domain
+    float *table_log2;     // tensor-core path, same memory: [batch * n_kv_heads][r_tot] -(max + log2 sum), log2 domain
     float *colsum;         // [n_kv_heads][sum_nv]
     float *mass;           // [sum_nv]
     WsHeader *header;
@@ -108,9 +109,9 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *res = base;                                  // [2] resident tiles: [chunk][128 rows][128 B], 128-byte swizzle
     uint8_t *ring = res + 2 * kTileBytes;                 // [kMassSlots] streamed tiles, same layout
-    float2 *tab = (float2 *)(ring + kMassSlots * kTileBytes);   // pass 1 only: (-max, 1 / sum) of the KV head's rows
-    const int tab_entries = PASS == 1 ? ((p.r_tot + 16 + 15) & ~15) : 0;
-    float2 *part = tab + tab_entries;                       // [2][kMassSlices][128]: the slices' partial results
+    float *tab = (float *)(ring + kMassSlots * kTileBytes);     // pass 1 only: -(max + log2 sum) of the KV head's rows
+    const int tab_entries = PASS == 1 ? ((p.r_tot + kMassSliceCols + 15) & ~15) : 0;
+    float2 *part = (float2 *)(tab + tab_entries);           // [2][kMassSlices][128]: the slices' partial results
     MassShared *sh = (MassShared *)(part + 2 * kMassSlices * kMassTile);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -156,8 +157,8 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
     // finite numbers: clear all tile buffers once.
     for (int x = tid; x < (2 + kMassSlots) * kTileBytes / 16; x += kMassThreads) reinterpret_cast<uint4 *>(res)[x] = make_uint4(0, 0, 0, 0);
     if (PASS == 1) {
-        const float2 *src = p.table + (size_t)unit * p.r_tot;
-        for (int x = tid; x < tab_entries; x += kMassThreads) tab[x] = x < p.r_tot ? src[x] : make_float2(0.f, 0.f);
+        const float *src = p.table_log2 + (size_t)unit * p.r_tot;
+        for (int x = tid; x < tab_entries; x += kMassThreads) tab[x] = x < p.r_tot ? src[x] : -INFINITY;
     }
     fence_proxy_async();
     tc_fence_before();
@@ -310,33 +311,31 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
                         }
                         l += add0 + add1;
                     } else {
-                        const float2 *tb = tab + i * TG + c0;
+                        // 2^(s * scale * log2e - max_r) / sum_r = 2^(s * sl2 + t_r): one table entry per column
+                        const float *tb = tab + i * TG + c0;
                         float a0 = 0.f, a1 = 0.f;
-                        if (mine == kMassSliceCols && ((i * TG) & 1) == 0) {
-                            // two table entries per 16-byte load (the block's first entry is 16-byte aligned)
+                        if (mine == kMassSliceCols && ((i * TG) & 3) == 0) {
                             float a2 = 0.f, a3 = 0.f;
-                            const float4 *tb4 = reinterpret_cast<const float4 *>(tb);
+                            const float4 *tb4 = reinterpret_cast<const float4 *>(tb);   // 16-byte aligned here
 #pragma unroll
                             for (int e = 0; e < kMassSliceCols; e += 4) {
-                                const float4 t0 = tb4[e >> 1], t1 = tb4[(e >> 1) + 1];
-                                a0 = fmaf(ex2_approx(fmaf(sv[e], sl2, t0.x)), t0.y, a0);
-                                a1 = fmaf(ex2_approx(fmaf(sv[e + 1], sl2, t0.z)), t0.w, a1);
-                                a2 = fmaf(ex2_approx(fmaf(sv[e + 2], sl2, t1.x)), t1.y, a2);
-                                a3 = fmaf(ex2_approx(fmaf(sv[e + 3], sl2, t1.z)), t1.w, a3);
+                                const float4 t = tb4[e >> 2];
+                                a0 += ex2_approx(fmaf(sv[e], sl2, t.x));
+                                a1 += ex2_approx(fmaf(sv[e + 1], sl2, t.y));
+                                a2 += ex2_approx(fmaf(sv[e + 2], sl2, t.z));
+                                a3 += ex2_approx(fmaf(sv[e + 3], sl2, t.w));
                             }
                             a0 += a2; a1 += a3;
                         } else if (mine == kMassSliceCols) {
 #pragma unroll
                             for (int e = 0; e < kMassSliceCols; e += 2) {
-                                const float2 t0 = tb[e], t1 = tb[e + 1];
-                                a0 = fmaf(ex2_approx(fmaf(sv[e], sl2, t0.x)), t0.y, a0);
-                                a1 = fmaf(ex2_approx(fmaf(sv[e + 1], sl2, t1.x)), t1.y, a1);
+                                a0 += ex2_approx(fmaf(sv[e], sl2, tb[e]));
+                                a1 += ex2_approx(fmaf(sv[e + 1], sl2, tb[e + 1]));
                             }
                         } else {
 #pragma unroll
                             for (int e = 0; e < kMassSliceCols; ++e) {
-                                const float2 t0 = tb[e];
-                                const float pe = ex2_approx(fmaf(sv[e], sl2, t0.x)) * t0.y;
+                                const float pe = ex2_approx(fmaf(sv[e], sl2, tb[e]));
                                 a0 += e < mine ? pe : 0.f;
                             }
                         }
@@ -381,7 +380,7 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
     }
 }
 
-// One thread per packed row of a KV head: merge the key splits of pass 1 into (-max, 1 / sum).
+// One thread per packed row of a KV head: merge the key splits of pass 1 into t = -(max + log2 sum).
 __global__ void mass_merge_kernel(const MassParams p) {
     const long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long total = (long long)p.batch * p.n_kv_heads * p.r_tot;
@@ -396,7 +395,7 @@ __global__ void mass_merge_kernel(const MassParams p) {
         const float2 v = src[(size_t)s * p.r_tot];
         if (v.y > 0.f) Lsum += v.y * exp2f(v.x - M);
     }
-    p.table[x] = Lsum > 0.f ? make_float2(-M, 1.f / Lsum) : make_float2(0.f, 0.f);
+    p.table_log2[x] = Lsum > 0.f ? -(M + log2f(Lsum)) : -INFINITY;
 }
 
 // mass += weight * (column sums of the KV heads, added in head order)
@@ -540,7 +539,7 @@ static int32_t launch_mass_tc(MassParams &p, const MassPlan &pl, long long pool_
     if (rc != HIPPO_OK) return rc;
     const size_t tiles = (size_t)(2 + kMassSlots) * kMassTile * D * 2;
     const size_t smem0 = 1024 + tiles + 2 * kMassSlices * kMassTile * sizeof(float2) + sizeof(MassShared) + 64;
-    const size_t smem1 = smem0 + (size_t)((p.r_tot + 16 + 15) & ~15) * sizeof(float2);
+    const size_t smem1 = smem0 + (size_t)((p.r_tot + kMassSliceCols + 15) & ~15) * sizeof(float);
     static PerDeviceOnce attr_set;
     int dev;
     if (attr_set.needed(dev)) {
@@ -633,6 +632,7 @@ extern "C" int32_t hippo_attention_mass(int32_t batch, const int32_t *n_visual, 
     p.page_table = kv->page_table; p.q = q_txt; p.k_pages = kv->k_pages;
     p.stats = (float2 *)((char *)workspace + pl.stats_off);
     p.table = (float2 *)((char *)workspace + pl.table_off);
+    p.table_log2 = (float *)p.table;
     p.colsum = (float *)((char *)workspace + pl.colsum_off);
     p.mass = mass;
     p.header = (WsHeader *)workspace;

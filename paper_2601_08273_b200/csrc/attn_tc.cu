@@ -946,15 +946,16 @@ bool attn_tc_supported(const AttnParams &p, int dtype) {
            p.rows <= kMaxRows;
 }
 
-// Cluster size for the one-cluster-per-unit mode, or 0 for the split modes.  `tiles` = upper bound of the tiles of a
+// Cluster size for the one-cluster-per-unit mode, or 0 for the split modes.  `pages` = upper bound of the pages of a
 // unit; max_active[cs] = clusters of cs CTAs of this kernel that the device keeps resident at once.  The cluster mode
 // needs no second kernel (worth about five tile times), but all clusters must be resident together and a unit gets
 // at most 16 SMs, so long caches with few units stay on the split path.
-static int choose_cluster_size(int units, int tiles, const int *max_active) {
-    int best = 0, best_cost = ceil_div(units * tiles, kNumSMs) + 5;
-    for (int cs = 2; cs <= 16 && cs <= tiles; ++cs) {
+static int choose_cluster_size(int units, int pages, const int *max_active) {
+    // costs in pages per CTA (ranges are cut on page boundaries); the second kernel of the split modes is worth ten
+    int best = 0, best_cost = ceil_div(units * pages, kNumSMs) + 10;
+    for (int cs = 2; cs <= 16 && 2 * cs <= pages + 1; ++cs) {
         if (units > max_active[cs]) continue;
-        const int cost = ceil_div(tiles, cs);
+        const int cost = ceil_div(pages, cs);
         if (cost < best_cost || (cost == best_cost && best == 0)) { best = cs; best_cost = cost; }
     }
     return best;
@@ -999,7 +1000,7 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
         }
         have_active[plan.slots].store(true, std::memory_order_release);
     }
-    const int cs = p.num_splits > 0 ? 0 : choose_cluster_size(units, ceil_div(p.max_kv_len, kBlockN), max_active[plan.slots]);
+    const int cs = p.num_splits > 0 ? 0 : choose_cluster_size(units, ceil_div(p.max_kv_len, kPageSize), max_active[plan.slots]);
     // Both kernels are launched with programmatic stream serialization and wait (griddepcontrol.wait) before they
     // touch memory, so stream order is kept while launch latency overlaps the previous kernel's tail.
     cudaLaunchAttribute attr[2];

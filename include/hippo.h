@@ -242,6 +242,69 @@ int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vocab, const 
                              const float *u_resample, int32_t mode, int32_t *n_accepted, int32_t *out_tokens,
                              void *stream);
 
+/* ---- decoding schedule: Section 5.2 (video parallel speculative decoding) -------------------------------------- */
+/*
+ * Host-only bookkeeping of the adaptive schedule; nothing here touches the GPU.  A round is planned, the caller
+ * launches what the plan says on its draft and verification streams, reads the accepted count back and commits it.
+ *   optimistic round   (previous batch accepted in full): verify the current batch (`verify_tokens` draft tokens,
+ *                      q_len = verify_tokens + 1) WHILE drafting the next `draft_during` = gamma tokens.  All accepted:
+ *                      the batch is emitted and the new tokens become the current batch.  Otherwise the accepted
+ *                      tokens and the target's replacement are emitted, the new tokens are dropped, and the next
+ *                      round is conservative.
+ *   conservative round (after a rejection): draft x_1 first (`draft_before` = 1), then verify x_1 WHILE drafting
+ *                      x_2..x_gamma (`draft_during` = gamma - 1).  x_1 rejected: stop drafting at once
+ *                      (`abort_on_reject`), emit the replacement, stay conservative.  x_1 accepted: emit it; the
+ *                      remaining tokens are the batch of an optimistic round (with gamma = 1 nothing remains: the
+ *                      target's bonus token is emitted too and the mode stays conservative).
+ * Synchronous draft-target prefill: the draft model keeps decoding while the target prefills;
+ * hippo_vpsd_prefill_buffer gives floor((prefill_target - prefill_draft) / t_draft) tokens, and a non-empty buffer
+ * handed to hippo_vpsd_init is the batch of a first optimistic round.
+ * The paper gives the two modes in words only; the emission and hand-over rules above are this library's reading.
+ */
+typedef enum hippo_vpsd_mode { HIPPO_VPSD_OPTIMISTIC = 0, HIPPO_VPSD_CONSERVATIVE = 1 } hippo_vpsd_mode_t;
+
+typedef struct hippo_vpsd_state {
+    uint32_t struct_size;       /* set by hippo_vpsd_init */
+    int32_t gamma;
+    int32_t mode;               /* hippo_vpsd_mode_t of the next round */
+    int32_t batch;              /* draft tokens waiting for verification at the start of the next round */
+    int64_t rounds;             /* statistics since init */
+    int64_t tokens_emitted;
+    int64_t tokens_drafted;
+    int64_t tokens_discarded;   /* drafted tokens that never reached the output */
+} hippo_vpsd_state_t;
+
+typedef struct hippo_vpsd_round {
+    int32_t mode;
+    int32_t draft_before;       /* draft tokens to produce before the verification starts */
+    int32_t verify_tokens;      /* draft tokens the target verifies this round */
+    int32_t draft_during;       /* draft tokens to produce while the target verifies */
+    int32_t abort_on_reject;    /* 1: stop drafting as soon as the verdict is a rejection */
+} hippo_vpsd_round_t;
+
+typedef struct hippo_vpsd_outcome {
+    int32_t accepted;           /* as committed */
+    int32_t emitted;            /* tokens appended to the output this round */
+    int32_t target_token;       /* 1: the last emitted token comes from the target (replacement or bonus) */
+    int32_t keep_drafted;       /* how many of the tokens drafted during the round form the next batch */
+    int32_t next_mode;
+} hippo_vpsd_outcome_t;
+
+/* All host pointers.  Status codes as everywhere; the two *_time functions return model time in the caller's unit. */
+int32_t hippo_vpsd_prefill_buffer(double prefill_target, double prefill_draft, double t_draft);
+int32_t hippo_vpsd_init(hippo_vpsd_state_t *state, int32_t gamma, int32_t buffered_tokens);
+int32_t hippo_vpsd_plan(const hippo_vpsd_state_t *state, hippo_vpsd_round_t *round);
+/* n_accepted in [0, verify_tokens]; drafted_during = tokens actually drafted beside the verification (less than
+ * round->draft_during only after an abort). */
+int32_t hippo_vpsd_commit(hippo_vpsd_state_t *state, const hippo_vpsd_round_t *round, int32_t n_accepted,
+                          int32_t drafted_during, hippo_vpsd_outcome_t *outcome);
+/* Duration of a round when one draft pass costs t_draft and one target pass t_target (the paper's latency
+ * example, Section 4.2, uses the same two constants): max(t_target, draft_during * t_draft) after the
+ * draft_before passes; a conservative round whose x_1 is rejected ends at the verdict. */
+double hippo_vpsd_round_time(const hippo_vpsd_round_t *round, int32_t n_accepted, double t_draft, double t_target);
+/* Serial speculative decoding for comparison: gamma draft passes, then one target pass (Section 4.2). */
+double hippo_vpsd_serial_round_time(int32_t gamma, double t_draft, double t_target);
+
 #ifdef __cplusplus
 }
 #endif

@@ -82,6 +82,39 @@ lib.hippo_accept_noalloc.restype = _i32
 lib.hippo_accept_noalloc.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
 ACCEPT_NOALLOC_SCRATCH_BYTES = 1024 * 1024
 
+HIPPO_VPSD_OPTIMISTIC = 0
+HIPPO_VPSD_CONSERVATIVE = 1
+_i64, _f64 = ctypes.c_int64, ctypes.c_double
+
+
+class VpsdState(ctypes.Structure):
+    _fields_ = [("struct_size", _u32), ("gamma", _i32), ("mode", _i32), ("batch", _i32), ("rounds", _i64),
+                ("tokens_emitted", _i64), ("tokens_drafted", _i64), ("tokens_discarded", _i64)]
+
+
+class VpsdRound(ctypes.Structure):
+    _fields_ = [("mode", _i32), ("draft_before", _i32), ("verify_tokens", _i32), ("draft_during", _i32),
+                ("abort_on_reject", _i32)]
+
+
+class VpsdOutcome(ctypes.Structure):
+    _fields_ = [("accepted", _i32), ("emitted", _i32), ("target_token", _i32), ("keep_drafted", _i32),
+                ("next_mode", _i32)]
+
+
+lib.hippo_vpsd_prefill_buffer.restype = _i32
+lib.hippo_vpsd_prefill_buffer.argtypes = [_f64, _f64, _f64]
+lib.hippo_vpsd_init.restype = _i32
+lib.hippo_vpsd_init.argtypes = [ctypes.POINTER(VpsdState), _i32, _i32]
+lib.hippo_vpsd_plan.restype = _i32
+lib.hippo_vpsd_plan.argtypes = [ctypes.POINTER(VpsdState), ctypes.POINTER(VpsdRound)]
+lib.hippo_vpsd_commit.restype = _i32
+lib.hippo_vpsd_commit.argtypes = [ctypes.POINTER(VpsdState), ctypes.POINTER(VpsdRound), _i32, _i32, ctypes.POINTER(VpsdOutcome)]
+lib.hippo_vpsd_round_time.restype = _f64
+lib.hippo_vpsd_round_time.argtypes = [ctypes.POINTER(VpsdRound), _i32, _f64, _f64]
+lib.hippo_vpsd_serial_round_time.restype = _f64
+lib.hippo_vpsd_serial_round_time.argtypes = [_i32, _f64, _f64]
+
 
 class HippoError(RuntimeError):
     def __init__(self, status: int):
@@ -260,6 +293,39 @@ def hippo_attention_mass(q_txt: torch.Tensor, kv: "KVCache", n_visual: Sequence[
                                     float(softmax_scale), float(weight), _ptr(mass), _ptr(workspace),
                                     workspace.numel(), _stream(stream)))
     return mass
+
+
+# ---- decoding schedule (Section 5.2), host only -------------------------------------------------------------------
+
+def hippo_vpsd_prefill_buffer(prefill_target: float, prefill_draft: float, t_draft: float) -> int:
+    return int(lib.hippo_vpsd_prefill_buffer(prefill_target, prefill_draft, t_draft))
+
+
+def hippo_vpsd_init(gamma: int, buffered_tokens: int = 0) -> VpsdState:
+    st = VpsdState()
+    _check(lib.hippo_vpsd_init(ctypes.byref(st), gamma, buffered_tokens))
+    return st
+
+
+def hippo_vpsd_plan(state: VpsdState) -> VpsdRound:
+    rd = VpsdRound()
+    _check(lib.hippo_vpsd_plan(ctypes.byref(state), ctypes.byref(rd)))
+    return rd
+
+
+def hippo_vpsd_commit(state: VpsdState, rnd: VpsdRound, n_accepted: int, drafted_during: Optional[int] = None) -> VpsdOutcome:
+    out = VpsdOutcome()
+    d = rnd.draft_during if drafted_during is None else drafted_during
+    _check(lib.hippo_vpsd_commit(ctypes.byref(state), ctypes.byref(rnd), int(n_accepted), int(d), ctypes.byref(out)))
+    return out
+
+
+def hippo_vpsd_round_time(rnd: VpsdRound, n_accepted: int, t_draft: float, t_target: float) -> float:
+    return float(lib.hippo_vpsd_round_time(ctypes.byref(rnd), int(n_accepted), t_draft, t_target))
+
+
+def hippo_vpsd_serial_round_time(gamma: int, t_draft: float, t_target: float) -> float:
+    return float(lib.hippo_vpsd_serial_round_time(gamma, t_draft, t_target))
 
 
 # ---- acceptance ---------------------------------------------------------------------------------------------------

@@ -1,0 +1,152 @@
+"""Decoding rounds of video parallel speculative decoding (Section 5.2) over the library's kernels.
+
+The schedule comes from the library's host-side scheduler (`hippo_vpsd_plan` / `hippo_vpsd_commit`); this module
+only launches what a round's plan says: draft attention calls on one CUDA stream, verification attention and
+`hippo_accept` on another, then one device-to-host read of the accepted count.  There are no models here: the query
+tensors and the logits are synthetic (seeded), positions do not advance (every round reads the same caches), and a
+"draft token" is `draft_layers` draft-attention calls.  What is real is the overlap pattern, the per-round
+verification length, the abort of a conservative round, and the acceptance kernel's verdicts that drive the mode
+switch.  Batch size 1, as in the paper.
+"""
+from __future__ import annotations
+
+import time
+from typing import Dict, List, Optional
+
+import torch
+
+from . import binding as hb
+from . import workloads as W
+from .step import HippoStep, _randn
+
+
+class VpsdLoop:
+    def __init__(self, cfg: W.HippoConfig, target_layers: Optional[int] = None, draft_layers: Optional[int] = None,
+                 buffered: int = 0, pool: int = 8, draft_noise: float = 1.0, device="cuda"):
+        assert cfg.batch == 1, "the schedule is per sequence; the driver runs one sequence"
+        self.cfg = cfg
+        self.st = HippoStep(cfg, device=device, target_layers=target_layers, draft_layers=draft_layers)
+        st, g = self.st, cfg.gamma
+        self.dev = st.device
+        self.max_batch = max(g, buffered)
+        G = cfg.tgt_q_heads // cfg.tgt_kv_heads
+        assert (self.max_batch + 1) * G <= 128, "verification batch exceeds the packed-row limit"
+        assert st.ctx[0] + self.max_batch + 1 <= st.tgt_cache[0].struct.max_pages_per_seq * hb.PAGE_SIZE, \
+            "the target cache has no room for the largest verification batch"
+        gen = torch.Generator(device=self.dev)
+        gen.manual_seed(3000 + cfg.seed)
+        mb = self.max_batch
+        # verification queries for up to max_batch + 1 rows; kv_len per batch size
+        self.q_t = _randn((st.Lt, 1, mb + 1, cfg.tgt_q_heads, cfg.tgt_head_dim), st.tdt, gen, self.dev)
+        self.out_t = torch.empty_like(self.q_t)
+        self.kv_len_t = {c: torch.tensor([st.ctx[0] + c + 1], dtype=torch.int32, device=self.dev) for c in range(1, mb + 1)}
+        self.verify_ws = hb.new_workspace(hb.hippo_attention_workspace_bytes(1, mb + 1, cfg.tgt_q_heads, cfg.tgt_kv_heads,
+                                                                             cfg.tgt_head_dim), self.dev)
+        # acceptance inputs: a pool of rounds; draft logits = target logits + noise, draft tokens drawn from them
+        V = cfg.vocab
+        self.pool = []
+        for _ in range(pool):
+            tl = torch.randn((1, mb + 1, V), device=self.dev, generator=gen) * cfg.logit_sigma
+            dl = tl[:, :mb] + draft_noise * torch.randn((1, mb, V), device=self.dev, generator=gen)
+            tok = torch.multinomial(torch.softmax(dl[0], dim=-1), 1, generator=gen).to(torch.int32).reshape(1, mb)
+            self.pool.append({"target_logits": tl.contiguous(), "draft_logits": dl.contiguous(), "draft_tokens": tok.contiguous(),
+                              "u_accept": torch.rand((1, mb), device=self.dev, generator=gen),
+                              "u_resample": torch.rand((1,), device=self.dev, generator=gen)})
+        self.n_accepted = torch.zeros(1, dtype=torch.int32, device=self.dev)
+        self.out_tokens = torch.empty((1, mb + 1), dtype=torch.int32, device=self.dev)
+        self.accept_ws = hb.new_workspace(hb.hippo_accept_workspace_bytes(1, mb, V), self.dev)
+        self.stream_d, self.stream_v = st.stream_d, st.stream_v
+
+    # ---- launches -------------------------------------------------------------------------------------------------
+    def draft_token(self, j: int, stream) -> None:
+        st = self.st
+        jj = j % self.cfg.gamma
+        for l in range(st.Ld):
+            hb.hippo_draft_attention(st.q_d[l, jj], st.dst_cache[l], st.kv_len_d[jj], st.max_kv_d[jj],
+                                     out=st.out_d[l, jj], workspace=st.draft_ws, stream=stream)
+
+    def verify_and_accept(self, c: int, pool_idx: int, stream) -> None:
+        st = self.st
+        for l in range(st.Lt):
+            hb.hippo_verify_attention(self.q_t[l][:, :c + 1], st.tgt_cache[l], self.kv_len_t[c], st.ctx[0] + c + 1,
+                                      out=self.out_t[l][:, :c + 1], workspace=self.verify_ws, stream=stream)
+        a = self.pool[pool_idx % len(self.pool)]
+        hb.hippo_accept(a["target_logits"][:, :c + 1], a["draft_logits"][:, :c], a["draft_tokens"][:, :c],
+                        a["u_accept"][:, :c], a["u_resample"], n_accepted=self.n_accepted,
+                        out_tokens=self.out_tokens[:, :c + 1], workspace=self.accept_ws, stream=stream)
+
+    # ---- the loops ----------------------------------------------------------------------------------------------------
+    def run(self, rounds: int, buffered: int = 0) -> Dict[str, object]:
+        """`rounds` rounds of the adaptive schedule.  Returns counters, the per-round trace and the wall time."""
+        state = hb.hippo_vpsd_init(self.cfg.gamma, buffered)
+        main = torch.cuda.current_stream(self.dev)
+        trace: List[dict] = []
+        torch.cuda.synchronize(self.dev)
+        t0 = time.perf_counter()
+        for r in range(rounds):
+            rd = hb.hippo_vpsd_plan(state)
+            for j in range(rd.draft_before):
+                self.draft_token(j, main)
+            self.stream_v.wait_stream(main)
+            self.stream_d.wait_stream(main)
+            self.verify_and_accept(rd.verify_tokens, r, self.stream_v)
+            verdict = torch.cuda.Event()
+            verdict.record(self.stream_v)
+            drafted, n = 0, None
+            for j in range(rd.draft_during):
+                if rd.abort_on_reject:
+                    # the host follows the drafting token by token and stops at a rejecting verdict
+                    if verdict.query():
+                        n = int(self.n_accepted.item())
+                        if n < rd.verify_tokens:
+                            break
+                self.draft_token(rd.draft_before + j, self.stream_d)
+                drafted += 1
+                if rd.abort_on_reject:
+                    self.stream_d.synchronize()
+            main.wait_stream(self.stream_v)
+            main.wait_stream(self.stream_d)
+            if n is None:
+                n = int(self.n_accepted.item())      # synchronises: the verdict is needed to plan the next round
+            if n == rd.verify_tokens and drafted < rd.draft_during:
+                for j in range(drafted, rd.draft_during):
+                    self.draft_token(rd.draft_before + j, main)
+                drafted = rd.draft_during
+            out = hb.hippo_vpsd_commit(state, rd, n, drafted)
+            trace.append({"mode": rd.mode, "batch": rd.verify_tokens, "accepted": n, "emitted": out.emitted,
+                          "drafted_during": drafted})
+        torch.cuda.synchronize(self.dev)
+        wall = time.perf_counter() - t0
+        return {"rounds": rounds, "tokens": int(state.tokens_emitted), "drafted": int(state.tokens_drafted),
+                "discarded": int(state.tokens_discarded), "wall_ms": wall * 1e3, "trace": trace}
+
+    def run_serial(self, rounds: int) -> Dict[str, object]:
+        """Serial speculative decoding for comparison: gamma draft tokens, then verification, on one stream."""
+        g = self.cfg.gamma
+        main = torch.cuda.current_stream(self.dev)
+        tokens = 0
+        torch.cuda.synchronize(self.dev)
+        t0 = time.perf_counter()
+        for r in range(rounds):
+            for j in range(g):
+                self.draft_token(j, main)
+            self.verify_and_accept(g, r, main)
+            tokens += int(self.n_accepted.item()) + 1
+        torch.cuda.synchronize(self.dev)
+        return {"rounds": rounds, "tokens": tokens, "wall_ms": (time.perf_counter() - t0) * 1e3}
+
+    def unit_times_ms(self, reps: int = 5) -> Dict[str, float]:
+        """One draft token and one verification pass (gamma tokens), each timed alone with CUDA events."""
+        main = torch.cuda.current_stream(self.dev)
+        def timed(fn):
+            fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(self.dev)
+            e0.record(main)
+            for _ in range(reps):
+                fn()
+            e1.record(main)
+            torch.cuda.synchronize(self.dev)
+            return e0.elapsed_time(e1) / reps
+        return {"t_draft": timed(lambda: self.draft_token(0, main)),
+                "t_target": timed(lambda: self.verify_and_accept(self.cfg.gamma, 0, main))}

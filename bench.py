@@ -383,6 +383,34 @@ def run_ours(args):
                 except Exception as e:  # noqa: BLE001
                     sweep.append({"gamma": g, "keep_pct": pct, "error": str(e)[:200]})
         extra.append({"workload": base.name + " sweep", "points": sweep})
+        # the adaptive decoding schedule (Section 5.2) over the kernels, against the serial schedule, on the bench workload
+        try:
+            from paper_2601_08273_b200.vpsd import VpsdLoop
+            torch.cuda.empty_cache()
+            loop = VpsdLoop(cfg, buffered=0, pool=8, draft_noise=0.5)
+            unit = loop.unit_times_ms()
+            loop.run(4); loop.run_serial(2)
+            par, ser = loop.run(60), loop.run_serial(30)
+            st8 = hb.hippo_vpsd_init(cfg.gamma, 0)
+            model_ms = 0.0
+            for t in par["trace"]:
+                rd = hb.hippo_vpsd_plan(st8)
+                model_ms += hb.hippo_vpsd_round_time(rd, t["accepted"], unit["t_draft"], unit["t_target"])
+                hb.hippo_vpsd_commit(st8, rd, t["accepted"], t["drafted_during"])
+            extra.append({"workload": cfg.name + " decoding schedule", "gamma": cfg.gamma, "rounds": par["rounds"],
+                          "t_draft_token_ms": unit["t_draft"], "t_verify_ms": unit["t_target"],
+                          "parallel_tokens": par["tokens"], "parallel_ms": par["wall_ms"],
+                          "parallel_tokens_per_s": par["tokens"] / par["wall_ms"] * 1e3,
+                          "parallel_model_ms": model_ms,
+                          "optimistic_rounds": sum(1 for t in par["trace"] if t["mode"] == 0),
+                          "mean_accepted": sum(t["accepted"] for t in par["trace"]) / par["rounds"],
+                          "serial_tokens": ser["tokens"], "serial_ms": ser["wall_ms"],
+                          "serial_tokens_per_s": ser["tokens"] / ser["wall_ms"] * 1e3,
+                          "note": "attention and acceptance kernels only, synthetic logits; host wall clock"})
+            del loop
+            torch.cuda.empty_cache()
+        except Exception as e:  # noqa: BLE001
+            extra.append({"workload": cfg.name + " decoding schedule", "error": str(e)[:200]})
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

@@ -22,7 +22,7 @@ from .step import HippoStep, _randn
 
 class VpsdLoop:
     def __init__(self, cfg: W.HippoConfig, target_layers: Optional[int] = None, draft_layers: Optional[int] = None,
-                 buffered: int = 0, pool: int = 8, draft_noise: float = 1.0, device="cuda"):
+                 buffered: int = 0, pool: int = 8, draft_noise: float = 1.0, use_graphs: bool = True, device="cuda"):
         assert cfg.batch == 1, "the schedule is per sequence; the driver runs one sequence"
         self.cfg = cfg
         self.st = HippoStep(cfg, device=device, target_layers=target_layers, draft_layers=draft_layers)
@@ -56,20 +56,56 @@ class VpsdLoop:
         self.out_tokens = torch.empty((1, mb + 1), dtype=torch.int32, device=self.dev)
         self.accept_ws = hb.new_workspace(hb.hippo_accept_workspace_bytes(1, mb, V), self.dev)
         self.stream_d, self.stream_v = st.stream_d, st.stream_v
+        # One draft token (draft_layers launches) and one verification pass (target_layers launches) are launch-bound
+        # when issued call by call from one host thread, which would serialise the two streams on the host: each is
+        # captured once into a CUDA graph and replayed.
+        self.g_draft = {}
+        self.g_verify = {}
+        if use_graphs:
+            for jj in range(g):
+                self.g_draft[jj] = self._capture(lambda s, jj=jj: self._draft_token_eager(jj, s))
+            for c in range(1, mb + 1):
+                self.g_verify[c] = self._capture(lambda s, c=c: self._verify_eager(c, s))
+
+    def _capture(self, fn):
+        side = torch.cuda.Stream(device=self.dev)
+        side.wait_stream(torch.cuda.current_stream(self.dev))
+        with torch.cuda.stream(side):
+            fn(side)                                   # warm-up: one-time set-up inside the library happens here
+        torch.cuda.current_stream(self.dev).wait_stream(side)
+        torch.cuda.synchronize(self.dev)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            fn(torch.cuda.current_stream(self.dev))
+        return graph
 
     # ---- launches -------------------------------------------------------------------------------------------------
-    def draft_token(self, j: int, stream) -> None:
+    def _draft_token_eager(self, jj: int, stream) -> None:
         st = self.st
-        jj = j % self.cfg.gamma
         for l in range(st.Ld):
             hb.hippo_draft_attention(st.q_d[l, jj], st.dst_cache[l], st.kv_len_d[jj], st.max_kv_d[jj],
                                      out=st.out_d[l, jj], workspace=st.draft_ws, stream=stream)
 
-    def verify_and_accept(self, c: int, pool_idx: int, stream) -> None:
+    def _verify_eager(self, c: int, stream) -> None:
         st = self.st
         for l in range(st.Lt):
             hb.hippo_verify_attention(self.q_t[l][:, :c + 1], st.tgt_cache[l], self.kv_len_t[c], st.ctx[0] + c + 1,
                                       out=self.out_t[l][:, :c + 1], workspace=self.verify_ws, stream=stream)
+
+    def draft_token(self, j: int, stream) -> None:
+        jj = j % self.cfg.gamma
+        if jj in self.g_draft:
+            with torch.cuda.stream(stream):
+                self.g_draft[jj].replay()
+        else:
+            self._draft_token_eager(jj, stream)
+
+    def verify_and_accept(self, c: int, pool_idx: int, stream) -> None:
+        if c in self.g_verify:
+            with torch.cuda.stream(stream):
+                self.g_verify[c].replay()
+        else:
+            self._verify_eager(c, stream)
         a = self.pool[pool_idx % len(self.pool)]
         hb.hippo_accept(a["target_logits"][:, :c + 1], a["draft_logits"][:, :c], a["draft_tokens"][:, :c],
                         a["u_accept"][:, :c], a["u_resample"], n_accepted=self.n_accepted,

@@ -53,3 +53,34 @@ def test_argument_validation_happens_before_any_launch():
     assert hb.hippo_select_workspace_bytes([100], 14, 14) >= 256 + 3 * 800
     assert hb.hippo_attention_workspace_bytes(1, 6, 28, 4, 128) > 42 * 130 * 4 * 4
     assert hb.hippo_accept_workspace_bytes(1, 5, 152064) > 0
+
+
+def test_attention_mass_argument_validation():
+    from paper_2601_08273_b200 import binding as hb
+    lib = hb.lib
+    kv = hb.KVCacheStruct(ctypes.sizeof(hb.KVCacheStruct), hb.HIPPO_DTYPE_BF16, 2, 128, 16, 8, 1024, 2048, None)
+    nv = (ctypes.c_int32 * 2)(300, 200)
+    need = lib.hippo_attention_mass_workspace_bytes(2, nv, 32, 8, 2, 128, hb.HIPPO_DTYPE_BF16)
+    assert need > 256
+    assert lib.hippo_attention_mass_workspace_bytes(2, nv, 32, 7, 2, 128, hb.HIPPO_DTYPE_BF16) == 0     # heads do not divide
+    assert lib.hippo_attention_mass_workspace_bytes(65, nv, 32, 8, 2, 128, hb.HIPPO_DTYPE_BF16) == 0    # batch limit
+    call = lambda **o: lib.hippo_attention_mass(o.get("B", 2), o.get("nv", nv), o.get("l_txt", 32), o.get("hq", 8), o.get("q", 256),
+                                                ctypes.byref(kv), ctypes.c_float(o.get("scale", 0.0)), ctypes.c_float(o.get("w", 1.0)),
+                                                o.get("mass", 256), o.get("ws", 256), o.get("ws_bytes", 1 << 30), None)
+    assert call(q=None) == hb.HIPPO_ERR_INVALID_ARG
+    assert call(hq=7) == hb.HIPPO_ERR_INVALID_ARG
+    assert call(B=65) == hb.HIPPO_ERR_UNSUPPORTED_SHAPE
+    assert call(ws_bytes=need - 1) == hb.HIPPO_ERR_WORKSPACE_TOO_SMALL
+    assert call(ws=264) == hb.HIPPO_ERR_INVALID_ARG                      # workspace alignment
+    assert call(scale=-1.0) == hb.HIPPO_ERR_INVALID_ARG
+    assert call(q=264 + 2) == hb.HIPPO_ERR_INVALID_ARG                   # query alignment
+    too_long = (ctypes.c_int32 * 2)(300, 8 * 64 + 1)
+    assert call(nv=too_long) == hb.HIPPO_ERR_INVALID_ARG                 # longer than the cache's pages
+    # identity page mapping needs batch * max_pages_per_seq <= n_pages: 2 * 8 = 16 fits, 3 sequences do not
+    nv3 = (ctypes.c_int32 * 3)(10, 10, 10)
+    assert call(B=3, nv=nv3) == hb.HIPPO_ERR_INVALID_ARG
+    # nothing to score: accepted, nothing launched
+    zero = (ctypes.c_int32 * 2)(0, 0)
+    before = hb.hippo_launch_count()
+    assert call(nv=zero) == hb.HIPPO_OK
+    assert hb.hippo_launch_count() == before

@@ -447,7 +447,12 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "kernel": "verify attention (%d launches per step)" % cfg.tgt_layers,
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": peak_src, "traffic": measured_traffic(cfg.name),
-                         "algorithmic_bytes_per_launch": kv_bytes_step // cfg.tgt_layers},
+                         "algorithmic_bytes_per_launch": kv_bytes_step // cfg.tgt_layers,
+                         # the same kernel (and the gather) on the longer workloads timed in this run, same peak
+                         "other_workloads": {e["workload"]: {"verify_gbps": round(e["verify_gbps"], 1),
+                                                             "verify_frac": round(e["verify_frac_of_measured_peak"], 3),
+                                                             "gather_frac": round(e["gather_frac_of_measured_peak"], 3)}
+                                             for e in extra if "verify_frac_of_measured_peak" in e}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches_per_step * steps + launches_per_verify_leg * steps),
             "gpu_launches_per_step": int(launches_per_step), "step_breakdown": breakdown, "extra": extra, "cpu_baseline": cpu,
         }

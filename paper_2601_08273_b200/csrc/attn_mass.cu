@@ -98,18 +98,27 @@ __device__ __forceinline__ bool mass_wait(MassShared *sh, WsHeader *hdr, unsigne
 }
 
 // PASS 0: row statistics (resident Q block, streamed key tiles).  PASS 1: column sums (resident key tile, streamed Q blocks).
+// Pass 0 keeps one resident tile and a ring of two, so that two CTAs share an SM: the maximum phase of one runs beside
+// the exponentials of the other.  Pass 1 changes its resident tile per outer step and double-buffers it.
+template <int PASS> struct MassBuffers {
+    static constexpr int kRes = PASS == 0 ? 1 : 2;
+    static constexpr int kSlots = PASS == 0 ? 2 : kMassSlots;
+    static constexpr int kCtasPerSm = PASS == 0 ? 2 : 1;
+};
+
 template <int D, int PASS>
-__global__ void __launch_bounds__(kMassThreads, 1)
+__global__ void __launch_bounds__(kMassThreads, MassBuffers<PASS>::kCtasPerSm)
 mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap q_map) {
     constexpr int kChunks = D / 64;                       // 64-column (128-byte) swizzle chunks per row
     constexpr int kChunkBytes = kMassTile * 128;          // one chunk of a 128-row tile
     constexpr int kTileBytes = kChunks * kChunkBytes;
     constexpr int kPageChunkBytes = kPageSize * 128;      // one chunk of one page
+    constexpr int kRes = MassBuffers<PASS>::kRes, kSlots = MassBuffers<PASS>::kSlots;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *res = base;                                  // [2] resident tiles: [chunk][128 rows][128 B], 128-byte swizzle
-    uint8_t *ring = res + 2 * kTileBytes;                 // [kMassSlots] streamed tiles, same layout
-    float *tab = (float *)(ring + kMassSlots * kTileBytes);     // pass 1 only: -(max + log2 sum) of the KV head's rows
+    uint8_t *ring = res + kRes * kTileBytes;              // [kSlots] streamed tiles, same layout
+    float *tab = (float *)(ring + kSlots * kTileBytes);   // pass 1 only: -(max + log2 sum) of the KV head's rows
     const int tab_entries = PASS == 1 ? ((p.r_tot + kMassSliceCols + 15) & ~15) : 0;
     float2 *part = (float2 *)(tab + tab_entries);           // [2][kMassSlices][128]: the slices' partial results
     MassShared *sh = (MassShared *)(part + 2 * kMassSlices * kMassTile);
@@ -137,8 +146,8 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
     }
 
     // ---- set-up
-    if (tid >= 32 && tid < 32 + kMassSlots) mbar_init(smem_u32(&sh->full[tid - 32]), 1);
-    else if (tid >= 40 && tid < 40 + kMassSlots) mbar_init(smem_u32(&sh->empty[tid - 40]), 1);
+    if (tid >= 32 && tid < 32 + kSlots) mbar_init(smem_u32(&sh->full[tid - 32]), 1);
+    else if (tid >= 40 && tid < 40 + kSlots) mbar_init(smem_u32(&sh->empty[tid - 40]), 1);
     else if (tid >= 48 && tid < 50) mbar_init(smem_u32(&sh->res_full[tid - 48]), 1);
     else if (tid >= 50 && tid < 52) mbar_init(smem_u32(&sh->res_free[tid - 50]), 1);
     else if (tid >= 52 && tid < 54) mbar_init(smem_u32(&sh->s_full[tid - 52]), 1);
@@ -155,7 +164,7 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
     }
     // Rows of a tile that no load ever writes (the last 128 - T*G rows of a Q block, a missing second page) must hold
     // finite numbers: clear all tile buffers once.
-    for (int x = tid; x < (2 + kMassSlots) * kTileBytes / 16; x += kMassThreads) reinterpret_cast<uint4 *>(res)[x] = make_uint4(0, 0, 0, 0);
+    for (int x = tid; x < (kRes + kSlots) * kTileBytes / 16; x += kMassThreads) reinterpret_cast<uint4 *>(res)[x] = make_uint4(0, 0, 0, 0);
     if (PASS == 1) {
         const float *src = p.table_log2 + (size_t)unit * p.r_tot;
         for (int x = tid; x < tab_entries; x += kMassThreads) tab[x] = x < p.r_tot ? src[x] : -INFINITY;
@@ -190,13 +199,13 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
             uint32_t issued = 0, res_issued = 0;
             bool ok = true;
             for (int o = o0; o < o1 && ok; ++o) {
-                const int rbuf = (o - o0) & 1;
-                ok = mass_wait(sh, hdr, &sh->res_free[rbuf], (((o - o0) >> 1) & 1) ^ 1, 1);
+                const int rbuf = (o - o0) % kRes;
+                ok = mass_wait(sh, hdr, &sh->res_free[rbuf], ((((o - o0) / kRes) & 1) ^ 1), 1);
                 if (!ok) break;
                 if (PASS == 0) load_rows(res + rbuf * kTileBytes, o, smem_u32(&sh->res_full[rbuf]));
                 else load_keys(res + rbuf * kTileBytes, o, smem_u32(&sh->res_full[rbuf]));
                 ++res_issued;
-                for (int i = i0; i < i1; ++i, rp.advance(kMassSlots), ++issued) {
+                for (int i = i0; i < i1; ++i, rp.advance(kSlots), ++issued) {
                     ok = mass_wait(sh, hdr, &sh->empty[rp.slot], rp.phase ^ 1, 2);
                     if (!ok) break;
                     if (PASS == 0) load_keys(ring + rp.slot * kTileBytes, i, smem_u32(&sh->full[rp.slot]));
@@ -204,13 +213,13 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
                 }
             }
             // every load that was issued must have landed before the CTA may exit
-            const int back = issued < (uint32_t)kMassSlots ? (int)issued : kMassSlots;
+            const int back = issued < (uint32_t)kSlots ? (int)issued : kSlots;
             for (int k = 0; k < back; ++k) {
-                if (rp.slot == 0) { rp.slot = kMassSlots - 1; rp.phase ^= 1; } else --rp.slot;
+                if (rp.slot == 0) { rp.slot = kSlots - 1; rp.phase ^= 1; } else --rp.slot;
                 mass_wait(sh, hdr, &sh->full[rp.slot], rp.phase, 3);
             }
-            for (uint32_t k = res_issued > 2 ? res_issued - 2 : 0; k < res_issued; ++k)
-                mass_wait(sh, hdr, &sh->res_full[k & 1], (k >> 1) & 1, 4);
+            for (uint32_t k = res_issued > (uint32_t)kRes ? res_issued - kRes : 0; k < res_issued; ++k)
+                mass_wait(sh, hdr, &sh->res_full[k % kRes], (k / kRes) & 1, 4);
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
@@ -222,9 +231,9 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
             uint32_t it = 0;
             bool ok = true;
             for (int o = o0; o < o1 && ok; ++o) {
-                const int rbuf = (o - o0) & 1;
-                ok = mass_wait(sh, hdr, &sh->res_full[rbuf], ((o - o0) >> 1) & 1, 5);
-                for (int i = i0; i < i1 && ok; ++i, ++it, rp.advance(kMassSlots)) {
+                const int rbuf = (o - o0) % kRes;
+                ok = mass_wait(sh, hdr, &sh->res_full[rbuf], ((o - o0) / kRes) & 1, 5);
+                for (int i = i0; i < i1 && ok; ++i, ++it, rp.advance(kSlots)) {
                     const int j = it & 1;
                     ok = mass_wait(sh, hdr, &sh->full[rp.slot], rp.phase, 6);
                     if (!ok) break;
@@ -468,11 +477,12 @@ struct MassPlan {
 
 // Key splits for `items` equal work items of `tiles` key tiles each (every key tile costing `inner` accumulator
 // tiles): the CTAs run one per SM in waves, so the cost is waves x (accumulator tiles per CTA + a fixed start-up).
-static int mass_best_splits(int items, int tiles, int inner) {
+static int mass_best_splits(int items, int tiles, int inner, int ctas_per_sm) {
     int best = 1;
     long long best_cost = -1;
+    const int room = kNumSMs * ctas_per_sm;
     for (int s = 1; s <= tiles && s <= kMassMaxSplits; ++s) {
-        const long long waves = ((long long)items * s + kNumSMs - 1) / kNumSMs;
+        const long long waves = ((long long)items * s + room - 1) / room;
         const long long cost = waves * ((long long)ceil_div(tiles, s) * inner + 4);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
     }
@@ -493,8 +503,8 @@ static MassPlan mass_plan(int batch, const int32_t *n_visual, int l_txt, int n_q
     for (int b = 0; b < batch; ++b) { sum_nv += n_visual[b]; if (n_visual[b] > max_nv) max_nv = n_visual[b]; }
     pl.max_nkt = ceil_div(max_nv > 0 ? max_nv : 1, kMassTile);
     const int units = batch * n_kv_heads;
-    pl.stat_splits = pl.tc ? mass_best_splits(units * pl.RB, pl.max_nkt, 1) : 1;
-    pl.sum_splits = mass_best_splits(units, pl.max_nkt, pl.RB);
+    pl.stat_splits = pl.tc ? mass_best_splits(units * pl.RB, pl.max_nkt, 1, MassBuffers<0>::kCtasPerSm) : 1;
+    pl.sum_splits = mass_best_splits(units, pl.max_nkt, pl.RB, MassBuffers<1>::kCtasPerSm);
     pl.stats_off = kWsHeaderBytes;
     pl.table_off = align_up(pl.stats_off + (size_t)units * pl.stat_splits * pl.r_tot * sizeof(float2), 256);
     pl.colsum_off = align_up(pl.table_off + (size_t)units * pl.r_tot * sizeof(float2), 256);
@@ -537,9 +547,10 @@ static int32_t launch_mass_tc(MassParams &p, const MassPlan &pl, long long pool_
     if (rc != HIPPO_OK) return rc;
     rc = make_q_map(&qm, p.q, p.batch, p.l_txt, p.n_q_heads, D, p.group, pl.T);
     if (rc != HIPPO_OK) return rc;
-    const size_t tiles = (size_t)(2 + kMassSlots) * kMassTile * D * 2;
-    const size_t smem0 = 1024 + tiles + 2 * kMassSlices * kMassTile * sizeof(float2) + sizeof(MassShared) + 64;
-    const size_t smem1 = smem0 + (size_t)((p.r_tot + kMassSliceCols + 15) & ~15) * sizeof(float);
+    const size_t tile = (size_t)kMassTile * D * 2, fixed = 1024 + 2 * kMassSlices * kMassTile * sizeof(float2) + sizeof(MassShared) + 64;
+    const size_t smem0 = fixed + (MassBuffers<0>::kRes + MassBuffers<0>::kSlots) * tile;
+    const size_t smem1 = fixed + (MassBuffers<1>::kRes + MassBuffers<1>::kSlots) * tile +
+                         (size_t)((p.r_tot + kMassSliceCols + 15) & ~15) * sizeof(float);
     static PerDeviceOnce attr_set;
     int dev;
     if (attr_set.needed(dev)) {

@@ -383,6 +383,24 @@ def run_ours(args):
                 except Exception as e:  # noqa: BLE001
                     sweep.append({"gamma": g, "keep_pct": pct, "error": str(e)[:200]})
         extra.append({"workload": base.name + " sweep", "points": sweep})
+        # what the fused score does to the border bias of the attention mass: share of frame-border tokens among the
+        # kept ones, attention term alone against all three terms (synthetic analogue of the paper's token-distribution figure)
+        try:
+            import numpy as np
+            stb = HippoStep(cfg, target_layers=1, draft_layers=1)
+            nv0, k0 = stb.n_visual[0], stb.k[0]
+            border = W.is_boundary(cfg, nv0)
+            shares = {}
+            for name, mask in (("attention_only", 1), ("all_terms", 7)):
+                kept, _ = hb.hippo_select_tokens(stb.embeds, stb.attn_mass, stb.n_visual, stb.k, cfg.grid_h, cfg.grid_w,
+                                                 cfg.crop_h, cfg.crop_w, score_mask=mask)
+                torch.cuda.synchronize()
+                shares[name] = float(border[kept[:k0].cpu().numpy()].mean())
+            extra.append({"workload": cfg.name + " kept-token border share", "border_share_of_all_tokens": float(border.mean()),
+                          "kept": k0, **shares})
+            del stb
+        except Exception as e:  # noqa: BLE001
+            extra.append({"workload": cfg.name + " kept-token border share", "error": str(e)[:200]})
         # the adaptive decoding schedule (Section 5.2) over the kernels, against the serial schedule, on the bench workload
         try:
             from paper_2601_08273_b200.vpsd import VpsdLoop

@@ -141,7 +141,7 @@ static TcSmemPlan tc_smem_plan(int D, int Rp) {
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
-               const int Rp, const int n_slots, const int tmem_cols, const int cluster_size) {
+               const int Rp, const int n_slots, const int tmem_cols, const int cluster_size, const int spare_cols) {
     constexpr int kChunks = D / 64;                     // 64-column (128-byte) swizzle chunks per row
     constexpr int kPageBytes = kPageSize * D * 2;       // K or V of one page and head
     constexpr int kSlotBytes = 2 * kPageBytes;          // K or V of one tile
@@ -471,6 +471,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         const int quarter = warp & 3;
         const int c_first = ((warp - 2) >> 2) * 16;   // this warp's row groups: c_first, c_first + 32, ...
         const uint32_t flip_groups = (Rp >> 4) & 1;
+        const bool spare_l = spare_cols != 0;         // a second column set for the partial row sums
+        int l_sel = 0;                                // which set holds the current sums
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const int kk = quarter * 32 + lane;           // key inside the tile
         const bool d_active = (D == 128) || lane < 16;
@@ -537,11 +539,61 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                     fence_proxy_async();
                 }
                 ok = W.wait(&sh->s_full[j], (it >> 1) & 1, 9) && ok;
+                // P^T buffer j was last read by PV of tile it-2
+                if (it >= 2) ok = W.wait(&sh->pv_done[j], ((it - 2) >> 1) & 1, 11) && ok;
                 tc_fence_after();
-                // ---- pass 1: does any visible score exceed its row's reference by more than the threshold?
-                // (branch-free inside; the masked variant runs only for the last tiles of a sequence)
-                float excess = -INFINITY;
-                if (!tail) {
+                uint8_t *pk = p_s + j * p_bytes + kk * 16;
+                const bool first_tile = it == it0;
+                // P^T = 2^(s*scale*log2e - reference) as bf16, row-contiguous per key, and the partial row sums
+                // (read from column set l_src unless this is the segment's first tile, written to l_dst).  Returns the
+                // largest exponent seen among the visible scores.  Branch-free inside; the masked variant runs only
+                // for the last tiles of a sequence.
+                auto write_p = [&](uint32_t l_src, uint32_t l_dst) -> float {
+                    float xmax = -INFINITY;
+                    for (int c = c_tile; c < Rp; c += 32) {
+                        float sv[16], lv[16];
+                        tmem_ld16(s_addr + c, sv);
+                        if (!first_tile) tmem_ld16(tmem + lane_addr + l_src + c, lv);
+                        tmem_wait_ld();
+                        uint32_t w[8];
+#pragma unroll
+                        for (int e4 = 0; e4 < 4; ++e4) {
+                            const float4 mn = *reinterpret_cast<const float4 *>(&sh->mneg[c + 4 * e4]);
+                            float x0 = fmaf(sv[4 * e4], sl2, mn.x), x1 = fmaf(sv[4 * e4 + 1], sl2, mn.y);
+                            float x2 = fmaf(sv[4 * e4 + 2], sl2, mn.z), x3 = fmaf(sv[4 * e4 + 3], sl2, mn.w);
+                            if (tail) {   // uniform over the CTA
+                                const int4 lm = *reinterpret_cast<const int4 *>(&sh->limit[c + 4 * e4]);
+                                x0 = key <= lm.x ? x0 : -INFINITY; x1 = key <= lm.y ? x1 : -INFINITY;
+                                x2 = key <= lm.z ? x2 : -INFINITY; x3 = key <= lm.w ? x3 : -INFINITY;
+                            }
+                            xmax = fmaxf(xmax, fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)));
+                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1), h1 = __floats2bfloat162_rn(p2, p3);
+                            w[2 * e4] = *reinterpret_cast<uint32_t *>(&h0);
+                            w[2 * e4 + 1] = *reinterpret_cast<uint32_t *>(&h1);
+                            if (first_tile) { lv[4 * e4] = p0; lv[4 * e4 + 1] = p1; lv[4 * e4 + 2] = p2; lv[4 * e4 + 3] = p3; }
+                            else { lv[4 * e4] += p0; lv[4 * e4 + 1] += p1; lv[4 * e4 + 2] += p2; lv[4 * e4 + 3] += p3; }
+                        }
+                        tmem_st16(tmem + lane_addr + l_dst + c, lv);
+                        *reinterpret_cast<uint4 *>(pk + (c >> 3) * (kBlockN * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4 *>(pk + ((c >> 3) + 1) * (kBlockN * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+                    }
+                    return xmax;
+                };
+                // ---- does any visible score exceed its row's reference by more than the threshold?
+                // With a spare column set for the row sums the answer comes out of the P^T pass itself, run on the
+                // stale references: if nothing grew (the common case) the tile is done after one sweep over S^T;
+                // otherwise the sweep is repeated below with the new references.  Without the spare set a cheaper
+                // sweep (maxima only) runs first.  The first tile of a segment always takes the slow path.
+                const uint32_t l_cur = col_l + l_sel * Rp, l_alt = spare_l ? col_l + (l_sel ^ 1) * Rp : l_cur;
+                float excess = NAN;
+                if (spare_l) {
+                    if (!first_tile) {
+                        excess = write_p(l_cur, l_alt);
+                        tmem_wait_st();
+                    }
+                } else if (!tail) {
+                    excess = -INFINITY;
                     for (int c = c_tile; c < Rp; c += 32) {
                         float sv[16];
                         tmem_ld16(s_addr + c, sv);
@@ -554,6 +606,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                         }
                     }
                 } else {
+                    excess = -INFINITY;
                     for (int c = c_tile; c < Rp; c += 32) {
                         float sv[16];
                         tmem_ld16(s_addr + c, sv);
@@ -569,8 +622,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                         }
                     }
                 }
-                // a NaN excess (inf - inf on a row that has seen nothing) must count as growth
+                // a NaN excess (inf - inf on a row that has seen nothing; the first tile) must count as growth
                 const bool grow = !(excess <= kRescaleThreshold);
+                tc_fence_before();
                 const bool any_grow = softmax_bar_or(grow || !ok);
                 tc_fence_after();   // the partial sums of this tile's columns may be the other warp's stores
                 if (sh->abort) { aborted = true; break; }
@@ -618,46 +672,25 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                         for (int c = c_tile; c < Rp; c += 32) {
                             float ov[16], lv[16];
                             tmem_ld16(tmem + lane_addr + col_o + c, ov);
-                            tmem_ld16(tmem + lane_addr + col_l + c, lv);
+                            tmem_ld16(tmem + lane_addr + l_cur + c, lv);
                             tmem_wait_ld();
 #pragma unroll
                             for (int e = 0; e < 16; ++e) { const float f = sh->fscale[c + e]; ov[e] *= f; lv[e] *= f; }
                             tmem_st16(tmem + lane_addr + col_o + c, ov);
-                            tmem_st16(tmem + lane_addr + col_l + c, lv);
+                            tmem_st16(tmem + lane_addr + l_cur + c, lv);
                         }
                         tmem_wait_st();
                     }
                 }
-                // ---- pass 2: P^T = 2^(s*scale*log2e - reference) as bf16, row-contiguous per key; partial row sums
-                // P^T buffer j was last read by PV of tile it-2
-                if (it >= 2) ok = W.wait(&sh->pv_done[j], ((it - 2) >> 1) & 1, 11) && ok;
-                uint8_t *pk = p_s + j * p_bytes + kk * 16;
-                const bool first_tile = it == it0;
-                for (int c = c_tile; c < Rp; c += 32) {
-                    float sv[16], lv[16];
-                    tmem_ld16(s_addr + c, sv);
-                    if (!first_tile) tmem_ld16(tmem + lane_addr + col_l + c, lv);
-                    tmem_wait_ld();
-                    uint32_t w[8];
-#pragma unroll
-                    for (int e4 = 0; e4 < 4; ++e4) {
-                        const float4 mn = *reinterpret_cast<const float4 *>(&sh->mneg[c + 4 * e4]);
-                        float p0 = ex2_approx(fmaf(sv[4 * e4], sl2, mn.x)), p1 = ex2_approx(fmaf(sv[4 * e4 + 1], sl2, mn.y));
-                        float p2 = ex2_approx(fmaf(sv[4 * e4 + 2], sl2, mn.z)), p3 = ex2_approx(fmaf(sv[4 * e4 + 3], sl2, mn.w));
-                        if (tail) {   // uniform over the CTA
-                            const int4 lm = *reinterpret_cast<const int4 *>(&sh->limit[c + 4 * e4]);
-                            p0 = key <= lm.x ? p0 : 0.f; p1 = key <= lm.y ? p1 : 0.f;
-                            p2 = key <= lm.z ? p2 : 0.f; p3 = key <= lm.w ? p3 : 0.f;
-                        }
-                        __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1), h1 = __floats2bfloat162_rn(p2, p3);
-                        w[2 * e4] = *reinterpret_cast<uint32_t *>(&h0);
-                        w[2 * e4 + 1] = *reinterpret_cast<uint32_t *>(&h1);
-                        if (first_tile) { lv[4 * e4] = p0; lv[4 * e4 + 1] = p1; lv[4 * e4 + 2] = p2; lv[4 * e4 + 3] = p3; }
-                        else { lv[4 * e4] += p0; lv[4 * e4 + 1] += p1; lv[4 * e4 + 2] += p2; lv[4 * e4 + 3] += p3; }
-                    }
-                    tmem_st16(tmem + lane_addr + col_l + c, lv);
-                    *reinterpret_cast<uint4 *>(pk + (c >> 3) * (kBlockN * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-                    *reinterpret_cast<uint4 *>(pk + ((c >> 3) + 1) * (kBlockN * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+                // ---- P^T and the row sums with the references that now hold
+                if (!spare_l || any_grow) (void)write_p(l_cur, l_alt);
+                l_sel ^= spare_l ? 1 : 0;
+                if (spare_l && any_grow && flip_groups) {
+                    // the next tile's sweep reads these sums from the other warp of the quarter before any barrier
+                    tmem_wait_st();
+                    tc_fence_before();
+                    softmax_bar_sync();
+                    tc_fence_after();
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -670,7 +703,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
             // (each warp sums the columns it stored itself in the segment's last tile)
             for (int c = c_first ^ ((int)((it - 1) & flip_groups) << 4); c < Rp; c += 32) {
                 float lv[16];
-                tmem_ld16(tmem + lane_addr + col_l + c, lv);
+                tmem_ld16(tmem + lane_addr + col_l + l_sel * Rp + c, lv);
                 tmem_wait_ld();
                 float mine = 0.f;
 #pragma unroll
@@ -972,8 +1005,10 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     const int Rp = (p.rows + 15) & ~15;
     const TcSmemPlan plan = tc_smem_plan(D, Rp);
     if (plan.slots < 3) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "attention: shared memory too small for %d packed rows", p.rows);
+    // tensor-memory columns: S^T x 2, O^T, partial row sums; a second set of sums when 512 columns allow it
+    const int spare_cols = 5 * Rp <= 512 ? Rp : 0;
     int tmem_cols = 32;
-    while (tmem_cols < 4 * Rp) tmem_cols *= 2;
+    while (tmem_cols < 4 * Rp + spare_cols) tmem_cols *= 2;
     static PerDeviceOnce attr_set;
     int dev;
     if (attr_set.needed(dev)) {
@@ -1020,7 +1055,7 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
         cfg.numAttrs = 2;
         cfg.gridDim = dim3((unsigned)(units * cs));
         if (slot_float_count(p.rows, D) * sizeof(float) <= (size_t)plan.slots * kBlockN * D * 2 &&
-            cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols, cs) == cudaSuccess) {
+            cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols, cs, spare_cols) == cudaSuccess) {
             count_launches(1);
             return HIPPO_OK;
         }
@@ -1028,7 +1063,7 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     }
     cfg.numAttrs = 1;
     cfg.gridDim = dim3((unsigned)grid);
-    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols, 0));
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, km, vm, Rp, plan.slots, tmem_cols, 0, spare_cols));
     count_launches(1);
     cfg.gridDim = dim3((unsigned)(p.batch * p.q_len * p.n_q_heads));
     cfg.blockDim = dim3(kCombineThreads);

@@ -53,6 +53,7 @@ class VpsdLoop:
                               "u_accept": torch.rand((1, mb), device=self.dev, generator=gen),
                               "u_resample": torch.rand((1,), device=self.dev, generator=gen)})
         self.n_accepted = torch.zeros(1, dtype=torch.int32, device=self.dev)
+        self.n_host = torch.zeros(1, dtype=torch.int32).pin_memory()
         self.out_tokens = torch.empty((1, mb + 1), dtype=torch.int32, device=self.dev)
         self.accept_ws = hb.new_workspace(hb.hippo_accept_workspace_bytes(1, mb, V), self.dev)
         self.stream_d, self.stream_v = st.stream_d, st.stream_v
@@ -112,42 +113,50 @@ class VpsdLoop:
                         out_tokens=self.out_tokens[:, :c + 1], workspace=self.accept_ws, stream=stream)
 
     # ---- the loops ----------------------------------------------------------------------------------------------------
+    def _verdict(self, c: int, pool_idx: int, stream, event) -> None:
+        """Verification of c draft tokens, acceptance, and the accepted count on its way to pinned host memory."""
+        self.verify_and_accept(c, pool_idx, stream)
+        with torch.cuda.stream(stream):
+            self.n_host.copy_(self.n_accepted, non_blocking=True)
+        event.record(stream)
+
     def run(self, rounds: int, buffered: int = 0) -> Dict[str, object]:
-        """`rounds` rounds of the adaptive schedule.  Returns counters, the per-round trace and the wall time."""
+        """`rounds` rounds of the adaptive schedule.  Returns counters, the per-round trace and the wall time.
+
+        The host touches a round twice: it launches what the plan says on the two streams, and it waits for the
+        verdict (one event, four bytes in pinned memory).  The verification stream waits on the device for the draft
+        tokens it verifies; nothing else is joined."""
         state = hb.hippo_vpsd_init(self.cfg.gamma, buffered)
-        main = torch.cuda.current_stream(self.dev)
+        sd, sv = self.stream_d, self.stream_v
+        verdict, batch_ready = torch.cuda.Event(), torch.cuda.Event()
         trace: List[dict] = []
         torch.cuda.synchronize(self.dev)
         t0 = time.perf_counter()
+        batch_ready.record(sd)                      # a prefill buffer is there from the start
         for r in range(rounds):
             rd = hb.hippo_vpsd_plan(state)
             for j in range(rd.draft_before):
-                self.draft_token(j, main)
-            self.stream_v.wait_stream(main)
-            self.stream_d.wait_stream(main)
-            self.verify_and_accept(rd.verify_tokens, r, self.stream_v)
-            verdict = torch.cuda.Event()
-            verdict.record(self.stream_v)
+                self.draft_token(j, sd)
+            if rd.draft_before:
+                batch_ready.record(sd)
+            sv.wait_event(batch_ready)              # the tokens to verify have been drafted
+            self._verdict(rd.verify_tokens, r, sv, verdict)
             drafted, n = 0, None
             for j in range(rd.draft_during):
                 if rd.abort_on_reject:
                     # the host follows the drafting token by token and stops at a rejecting verdict
                     if verdict.query():
-                        n = int(self.n_accepted.item())
+                        n = int(self.n_host[0])
                         if n < rd.verify_tokens:
                             break
-                self.draft_token(rd.draft_before + j, self.stream_d)
+                self.draft_token(rd.draft_before + j, sd)
                 drafted += 1
                 if rd.abort_on_reject:
-                    self.stream_d.synchronize()
-            main.wait_stream(self.stream_v)
-            main.wait_stream(self.stream_d)
+                    sd.synchronize()
+            batch_ready.record(sd)
             if n is None:
-                n = int(self.n_accepted.item())      # synchronises: the verdict is needed to plan the next round
-            if n == rd.verify_tokens and drafted < rd.draft_during:
-                for j in range(drafted, rd.draft_during):
-                    self.draft_token(rd.draft_before + j, main)
-                drafted = rd.draft_during
+                verdict.synchronize()               # the verdict is needed to plan the next round
+                n = int(self.n_host[0])
             out = hb.hippo_vpsd_commit(state, rd, n, drafted)
             trace.append({"mode": rd.mode, "batch": rd.verify_tokens, "accepted": n, "emitted": out.emitted,
                           "drafted_during": drafted})
@@ -160,14 +169,16 @@ class VpsdLoop:
         """Serial speculative decoding for comparison: gamma draft tokens, then verification, on one stream."""
         g = self.cfg.gamma
         main = torch.cuda.current_stream(self.dev)
+        verdict = torch.cuda.Event()
         tokens = 0
         torch.cuda.synchronize(self.dev)
         t0 = time.perf_counter()
         for r in range(rounds):
             for j in range(g):
                 self.draft_token(j, main)
-            self.verify_and_accept(g, r, main)
-            tokens += int(self.n_accepted.item()) + 1
+            self._verdict(g, r, main, verdict)
+            verdict.synchronize()
+            tokens += int(self.n_host[0]) + 1
         torch.cuda.synchronize(self.dev)
         return {"rounds": rounds, "tokens": tokens, "wall_ms": (time.perf_counter() - t0) * 1e3}
 

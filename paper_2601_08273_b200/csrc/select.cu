@@ -322,7 +322,9 @@ __device__ __forceinline__ uint32_t order_key(float x) {  // larger float -> lar
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-__global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p) {
+// smem_keys: keys beyond the 32 per thread that live in registers are staged in this many words of dynamic shared memory
+__global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p, const int smem_keys) {
+    extern __shared__ uint32_t skeys[];
     __shared__ int warp_cnt[32];
     __shared__ uint32_t s_prefix;
     __shared__ int s_remaining, s_base_eq, s_base_out;
@@ -333,39 +335,42 @@ __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p)
     const float *score = p.fused + p.seq_off[b];
     int32_t *out = p.kept + p.k_off[b];
     // The key T of the k-th largest element, two bits at a time from the top: T is the largest value with at least k
-    // keys >= T.  Each thread keeps its keys in registers (up to 32 per thread; longer sequences are read again from
-    // memory), so a step is a few compares and one block-wide sum of three counters.
+    // keys >= T.  Each thread keeps its keys in registers (32 per thread), the next ones in shared memory, and only
+    // what is left beyond both is read again from memory, so a step is a few compares and one block-wide sum of three
+    // counters.
     constexpr int kKeysPerThread = 32;
     __shared__ int warp_cnt3[32][3];
     __shared__ int s_cnt3[3];
     uint32_t keys[kKeysPerThread];
-    const bool in_regs = n <= kKeysPerThread * (int)blockDim.x;
-    if (in_regs) {
+    const int n_regs = kKeysPerThread * (int)blockDim.x;            // keys [0, n_regs) in registers
+    const int n_staged = min(n, n_regs + smem_keys);                 // keys [n_regs, n_staged) in shared memory
 #pragma unroll
-        for (int e = 0; e < kKeysPerThread; ++e) {
-            const int i = e * blockDim.x + tid;
-            keys[e] = i < n ? order_key(score[i]) : 0u;   // padding: key 0 is never counted (candidates are > 0)
-        }
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        const int i = e * blockDim.x + tid;
+        keys[e] = i < n ? order_key(score[i]) : 0u;   // padding: key 0 is never counted (candidates are > 0)
     }
-    const int per_thread = (n + (int)blockDim.x - 1) / (int)blockDim.x;
+    for (int i = n_regs + tid; i < n_staged; i += blockDim.x) skeys[i - n_regs] = order_key(score[i]);
+    __syncthreads();
+    const int per_thread = min(kKeysPerThread, (n + (int)blockDim.x - 1) / (int)blockDim.x);
     // counts of keys >= c1, >= c2, >= c3 over the sequence (candidates are non-zero)
     auto count3 = [&](uint32_t c1, uint32_t c2, uint32_t c3) {
         int a1 = 0, a2 = 0, a3 = 0;
-        if (in_regs) {
 #pragma unroll
-            for (int e0 = 0; e0 < kKeysPerThread; e0 += 8) {
-                if (e0 < per_thread) {      // uniform: only the groups of eight that hold keys
+        for (int e0 = 0; e0 < kKeysPerThread; e0 += 8) {
+            if (e0 < per_thread) {      // uniform: only the groups of eight that hold keys
 #pragma unroll
-                    for (int e = e0; e < e0 + 8; ++e) {
-                        a1 += keys[e] >= c1 ? 1 : 0; a2 += keys[e] >= c2 ? 1 : 0; a3 += keys[e] >= c3 ? 1 : 0;
-                    }
+                for (int e = e0; e < e0 + 8; ++e) {
+                    a1 += keys[e] >= c1 ? 1 : 0; a2 += keys[e] >= c2 ? 1 : 0; a3 += keys[e] >= c3 ? 1 : 0;
                 }
             }
-        } else {
-            for (int i = tid; i < n; i += blockDim.x) {
-                const uint32_t key = order_key(score[i]);
-                a1 += key >= c1 ? 1 : 0; a2 += key >= c2 ? 1 : 0; a3 += key >= c3 ? 1 : 0;
-            }
+        }
+        for (int i = n_regs + tid; i < n_staged; i += blockDim.x) {
+            const uint32_t key = skeys[i - n_regs];
+            a1 += key >= c1 ? 1 : 0; a2 += key >= c2 ? 1 : 0; a3 += key >= c3 ? 1 : 0;
+        }
+        for (int i = n_staged + tid; i < n; i += blockDim.x) {
+            const uint32_t key = order_key(score[i]);
+            a1 += key >= c1 ? 1 : 0; a2 += key >= c2 ? 1 : 0; a3 += key >= c3 ? 1 : 0;
         }
         a1 = __reduce_add_sync(0xffffffffu, a1);
         a2 = __reduce_add_sync(0xffffffffu, a2);
@@ -539,7 +544,21 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
     const int fuse_threads = ((p.tpf + 31) / 32) * 32;
     select_fuse_kernel<<<(unsigned)frames, fuse_threads, 0, s>>>(p);
     count_launches(1);
-    if (ksum > 0) { select_topk_kernel<<<batch, 1024, 0, s>>>(p); count_launches(1); }
+    if (ksum > 0) {
+        // shared-memory staging for the keys beyond 32 per thread, up to 48K of them
+        int longest = 0;
+        for (int b = 0; b < batch; ++b) longest = n_visual[b] > longest ? n_visual[b] : longest;
+        int smem_keys = longest - 32 * 1024;
+        smem_keys = smem_keys < 0 ? 0 : (smem_keys > 48 * 1024 ? 48 * 1024 : smem_keys);
+        static PerDeviceOnce topk_attr;
+        int dev;
+        if (topk_attr.needed(dev)) {
+            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 48 * 1024 * 4));
+            topk_attr.mark(dev);
+        }
+        select_topk_kernel<<<batch, 1024, (size_t)smem_keys * 4, s>>>(p, smem_keys);
+        count_launches(1);
+    }
     HIPPO_CUDA_TRY(cudaGetLastError());
     return HIPPO_OK;
 }

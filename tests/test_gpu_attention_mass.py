@@ -139,3 +139,14 @@ def test_feeds_the_selection(hb):
     diff = np.setxor1d(host(kept)[:k], ref_kept)
     assert band[diff].all()
     assert len(diff) <= 8
+
+
+def test_reproducible_bits(hb):
+    """The sums run in a fixed order: the same call gives the same bits, whatever else the GPU did in between."""
+    cfg = W.CONFIGS[1]
+    nv = W.visual_lengths(cfg)
+    inp = W.mass_inputs(cfg, nv, layer=3)
+    a = gpu_mass(hb, [inp["q_txt"]], [inp["k_vid"]], nv, cfg.dtype)
+    torch.randn(1 << 22, device="cuda").sum().item()
+    b = gpu_mass(hb, [inp["q_txt"]], [inp["k_vid"]], nv, cfg.dtype)
+    np.testing.assert_array_equal(a, b)

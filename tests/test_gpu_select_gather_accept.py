@@ -119,6 +119,21 @@ def test_c4_select_sampled_frames(hb):
         assert kept.tolist() == want.tolist()
 
 
+def test_topk_all_three_key_tiers(hb):
+    """100,352 tokens: keys in registers, in shared memory and re-read from memory; many equal scores (attention term
+    only, mass quantised to 64 levels) so that the index tie-break decides most of the threshold."""
+    rng = np.random.default_rng(11)
+    n, d = 512 * 196, 8
+    E = dev(rng.standard_normal((n, d)).astype(np.float32))
+    mass = dev((rng.integers(0, 64, size=n) / 64.0).astype(np.float32))
+    for k in (1, 5000, 50177, n):
+        kept, fused = hb.hippo_select_tokens(E, mass, [n], [k], 14, 14, score_mask=1)
+        torch.cuda.synchronize()
+        kept, fused = host(kept), host(fused)
+        want = np.sort(np.lexsort((np.arange(n), -fused.astype(np.float64)))[:k])
+        assert kept.tolist() == want.tolist()
+
+
 # ---- gather -------------------------------------------------------------------------------------------------------
 
 def run_gather(hb, cfg, n_layers, src_lens, keeps, dtype, shuffle=(None, None)):

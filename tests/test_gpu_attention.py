@@ -82,6 +82,24 @@ def test_packed_row_shapes_bf16(hb, rows):
     check_full(hb, hb.hippo_verify_attention, q, k, v, lens, "bf16")
 
 
+
+@pytest.mark.parametrize("q_len,Hq,Hkv", [(6, 8, 2), (6, 14, 2), (9, 16, 2), (16, 16, 2)])
+def test_reference_maxima_keep_growing(hb, q_len, Hq, Hkv):
+    """Keys grow along the sequence, so that in tile after tile some scores exceed the rows' running maxima by far
+    more than the lazy-rescale threshold: the rescale path (and the repeated probability sweep) runs mid-sequence,
+    for 24, 42, 72 and 128 packed rows (with and without the spare row-sum columns, even and odd group counts)."""
+    rng = np.random.default_rng(23)
+    D, lens = 128, [1500, 700]
+    q = W.round_to_storage(2.0 * rng.standard_normal((2, q_len, Hq, D)).astype(np.float32), "bf16")
+    k = rng.standard_normal((2, max(lens), Hkv, D)).astype(np.float32)
+    k *= (1.0 + 2.0 * (np.arange(max(lens)) // 100))[None, :, None, None]
+    k[1, :, :, :] *= np.where(np.arange(max(lens)) % 257 == 0, 3.0, 1.0)[:, None, None]    # isolated spikes as well
+    k = W.round_to_storage(k, "bf16")
+    v = W.round_to_storage(rng.standard_normal((2, max(lens), Hkv, D)).astype(np.float32), "bf16")
+    check_full(hb, hb.hippo_verify_attention, q, k, v, lens, "bf16", shuffle_seed=3)
+    check_full(hb, hb.hippo_verify_attention, q, k, v, lens, "bf16", shuffle_seed=3, num_splits=3)
+
+
 @pytest.mark.parametrize("D", [64, 128])
 def test_more_units_than_sms(hb, D):
     """200 (sequence, kv head) units: more than one per SM, so CTAs walk several units and units straddle CTAs."""

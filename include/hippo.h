@@ -170,7 +170,9 @@ int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src, size_t sr
  * CTA per SM streaming K/V tiles); hippo_draft_attention for q_len = 1 against the short pruned cache
  * (many small splits).  Both compute the same function for any q_len >= 1.
  *   q        [batch][q_len][n_q_heads][head_dim] dtype        out  same shape and dtype as q
- *   kv_len   int32 [batch] (device), q_len <= kv_len[b] <= max_kv_len;  a sequence with kv_len[b] < q_len is skipped
+ *   kv_len   int32 [batch] (device), q_len <= kv_len[b] <= max_kv_len;  a sequence with kv_len[b] < q_len is skipped.
+ *            NULL means the lengths are known on the host and all equal max_kv_len: the kernels then start their
+ *            loads without the round trip for the length
  *   max_kv_len  host upper bound used to size the launch; <= max_pages_per_seq * 64
  *   softmax_scale  0 selects 1/sqrt(head_dim)
  *   num_splits  0 = automatic

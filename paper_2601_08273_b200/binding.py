@@ -245,7 +245,7 @@ def hippo_attention_workspace_bytes(batch: int, q_len: int, n_q_heads: int, n_kv
 
 
 def _attention(fn, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse, workspace, stream):
-    assert q.is_contiguous() and q.dim() == 4 and kv_len.dtype == torch.int32
+    assert q.is_contiguous() and q.dim() == 4 and (kv_len is None or kv_len.dtype == torch.int32)
     B, q_len, hq, d = q.shape
     assert d == kv.head_dim and _dtype_code(q) == kv.struct.dtype
     if out is None:

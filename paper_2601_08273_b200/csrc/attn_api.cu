@@ -27,7 +27,7 @@ static int32_t attention_entry(const char *who, bool draft_policy, int32_t batch
     if (rc != HIPPO_OK) return rc;
     if (batch <= 0 || q_len <= 0 || n_q_heads <= 0 || max_kv_len <= 0 || num_splits < 0)
         return fail(HIPPO_ERR_INVALID_ARG, "%s: non-positive size", who);
-    if (!q || !out || !kv_len || !workspace) return fail(HIPPO_ERR_INVALID_ARG, "%s: null pointer", who);
+    if (!q || !out || !workspace) return fail(HIPPO_ERR_INVALID_ARG, "%s: null pointer", who);
     if (n_q_heads % kv->n_kv_heads) return fail(HIPPO_ERR_INVALID_ARG, "%s: n_q_heads %% n_kv_heads != 0", who);
     if ((long long)batch * kv->n_kv_heads > 16000) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: batch*n_kv_heads > 16000", who);
     const int G = n_q_heads / kv->n_kv_heads, rows = q_len * G;

@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kGenThreads) attn_generic_kernel(const AttnPar
 
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int kvl = p.kv_len[b];
+    const int kvl = p.kv_len ? p.kv_len[b] : p.max_kv_len;
     float *slot = p.partials + ((size_t)(b * p.n_kv_heads + hk) * p.num_splits + split) * slot_float_count(R, D);
     const int Rp = slot_rows_padded(R);
     if (kvl < p.q_len) return;  // combine writes zeros for such sequences
@@ -107,7 +107,7 @@ __global__ void attn_combine_kernel(const AttnParams p, int n_splits) {
     const int h = row % p.n_q_heads, t = (row / p.n_q_heads) % p.q_len, b = row / (p.n_q_heads * p.q_len);
     const int hk = h / G, r = t * G + (h % G);
     T *out = (T *)p.out + (size_t)row * D;
-    if (p.kv_len[b] < p.q_len) {
+    if ((p.kv_len ? p.kv_len[b] : p.max_kv_len) < p.q_len) {
         for (int d = lane; d < D; d += 32) store_from_float(out + d, 0.f);
         if (p.lse && lane == 0) p.lse[row] = -INFINITY;
         return;

@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(kSmThreads) attn_small_kernel(const AttnParams
     const int R = p.rows, G = p.group, Hkv = p.n_kv_heads;
     const int unit = blockIdx.x / cluster_size, rank = blockIdx.x % cluster_size;
     const int b = unit / Hkv, hk = unit % Hkv;
-    const int kvl = p.kv_len[b];
+    const int kvl = p.kv_len ? p.kv_len[b] : p.max_kv_len;   // no length array: every sequence has max_kv_len keys
     const bool skipped = kvl < p.q_len;
     const int n_pages = skipped ? 0 : (kvl + kSmPage - 1) / kSmPage;
     const int pg_begin = (int)((long long)n_pages * rank / cluster_size), pg_end = (int)((long long)n_pages * (rank + 1) / cluster_size);

@@ -190,13 +190,13 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
         if (!small_problem) {
             // tiles per sequence; the exclusive prefix follows the barrier
             for (int b = tid; b < B; b += kTcThreads) {
-                const int kvl = p.kv_len[b];
+                const int kvl = p.kv_len ? p.kv_len[b] : p.max_kv_len;
                 sh->kvlen[b] = kvl;
                 sh->tile_prefix[b + 1] = seq_tiles(kvl, p.q_len);
             }
         } else if (warp == 0) {
             // lane b: sequence b; lane u: unit u.  Everything by shuffles.
-            const int kvl = lane < B ? p.kv_len[lane] : 0;
+            const int kvl = lane < B ? (p.kv_len ? p.kv_len[lane] : p.max_kv_len) : 0;
             const int nt = lane < B ? seq_tiles(kvl, p.q_len) : 0;
             int incl = nt;
 #pragma unroll

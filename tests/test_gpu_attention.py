@@ -202,6 +202,26 @@ def test_full_size_draft(hb, ci):
         assert_close(got, ref, TOL[cfg.dtype], "c%d draft keep %d%%" % (ci, pct))
 
 
+@pytest.mark.parametrize("dtype,q_len,kvl", [("bf16", 6, 700), ("bf16", 1, 500), ("fp32", 3, 200)])
+def test_lengths_known_on_the_host(hb, dtype, q_len, kvl):
+    """kv_len = NULL: every sequence has max_kv_len keys; same result as with the length array."""
+    rng = np.random.default_rng(31)
+    B, Hq, Hkv, D = 2, 8, 2, 64
+    lens = [kvl, kvl]
+    q = W.round_to_storage(rng.standard_normal((B, q_len, Hq, D)).astype(np.float32), dtype)
+    k = W.round_to_storage(rng.standard_normal((B, kvl, Hkv, D)).astype(np.float32), dtype)
+    v = W.round_to_storage(rng.standard_normal((B, kvl, Hkv, D)).astype(np.float32), dtype)
+    kv, _, _ = paged_cache(hb, k, v, lens, dtype, shuffle_seed=2)
+    with_array = host(hb.hippo_verify_attention(dev(q, dtype), kv, dev(np.asarray(lens, np.int32)), kvl))
+    without = host(hb.hippo_verify_attention(dev(q, dtype), kv, None, kvl))
+    draft = host(hb.hippo_draft_attention(dev(q, dtype), kv, None, kvl))
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(with_array, without)
+    ref, _ = oracle.attention(q, k, v, lens)
+    assert_close(without, ref, TOL[dtype], "host lengths")
+    assert_close(draft, ref, TOL[dtype], "host lengths, draft")
+
+
 def test_workspace_status_is_clean(hb):
     ws = hb.new_workspace(hb.hippo_attention_workspace_bytes(1, 2, 4, 2, 64))
     rng = np.random.default_rng(0)

@@ -77,6 +77,39 @@ struct Partition {
 // 128-key tiles from consecutive pairs of its pages (the last tile of a range may hold a single page).
 __device__ __forceinline__ int seq_tiles(int kvl, int q_len) { return kvl < q_len ? 0 : (kvl + kPageSize - 1) / kPageSize; }
 
+// Unit-aligned split worked out by one warp (at most 32 units): every unit with tiles gets one CTA, the others go to
+// the units in proportion to their tile counts (largest remainders first, lower unit first on ties), never more CTAs
+// than tiles.  Lane u holds unit u: my_tiles = its tiles (0 beyond the last unit), total = tiles of all units.
+// Returns (first CTA, CTAs) of the lane's unit; all_ctas = CTAs in use.  The main kernel and the combine kernel both
+// call this, so they cannot disagree.
+__device__ __forceinline__ int2 aligned_split_warp(int lane, int U, int grid, int my_tiles, long long total, int &all_ctas) {
+    const bool live = my_tiles > 0;
+    const int spare = grid - __popc(__ballot_sync(0xffffffffu, live));
+    int base = 0;
+    uint32_t r = 0;
+    if (live) {
+        const long long num = (long long)spare * my_tiles;
+        base = (int)(num / total);
+        r = (uint32_t)(num % total);
+    }
+    int sum_base = base;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) sum_base += __shfl_xor_sync(0xffffffffu, sum_base, o);
+    const int leftover = spare - sum_base;
+    int rank = 0;
+    for (int v = 0; v < U; ++v) {
+        const uint32_t rv = __shfl_sync(0xffffffffu, r, v);
+        const int lv = __shfl_sync(0xffffffffu, (int)live, v);
+        rank += (lv && (rv > r || (rv == r && v < lane))) ? 1 : 0;
+    }
+    const int n = live ? min(my_tiles, 1 + base + (rank < leftover ? 1 : 0)) : 0;
+    int cinc = n;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, cinc, o); if (lane >= o) cinc += v; }
+    all_ctas = __shfl_sync(0xffffffffu, cinc, 31);
+    return make_int2(cinc - n, n);
+}
+
 // ---- shared control block -------------------------------------------------------------------------------------------
 struct TcShared {
     unsigned long long full[kMaxSlots], empty[kMaxSlots], s_full[2], s_free[2], p_full[2], pv_done[2], q_full, q_free, drain;
@@ -208,31 +241,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
                 const long long total = (long long)__shfl_sync(0xffffffffu, incl, 31) * Hkv;
                 const int t_src = __shfl_sync(0xffffffffu, nt, lane < U ? lane / Hkv : 0);
                 const int my_tiles = lane < U ? t_src : 0;
-                const bool live = my_tiles > 0;
-                const int spare = (int)gridDim.x - __popc(__ballot_sync(0xffffffffu, live));
-                int base = 0;
-                uint32_t r = 0;
-                if (live) {
-                    const long long num = (long long)spare * my_tiles;
-                    base = (int)(num / total);
-                    r = (uint32_t)(num % total);
-                }
-                int sum_base = base;
-#pragma unroll
-                for (int o = 16; o; o >>= 1) sum_base += __shfl_xor_sync(0xffffffffu, sum_base, o);
-                const int leftover = spare - sum_base;
-                int rank = 0;
-                for (int v = 0; v < U; ++v) {
-                    const uint32_t rv = __shfl_sync(0xffffffffu, r, v);
-                    const int lv = __shfl_sync(0xffffffffu, (int)live, v);
-                    rank += (lv && (rv > r || (rv == r && v < lane))) ? 1 : 0;
-                }
-                const int n = live ? min(my_tiles, 1 + base + (rank < leftover ? 1 : 0)) : 0;
-                int cinc = n;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, cinc, o); if (lane >= o) cinc += v; }
-                if (lane < U) { sh->n_cta[lane] = n; sh->cta_base[lane] = cinc - n; }
-                const int all = __shfl_sync(0xffffffffu, cinc, 31);
+                int all;
+                const int2 mine = aligned_split_warp(lane, U, (int)gridDim.x, my_tiles, total, all);
+                if (lane < U) { sh->n_cta[lane] = mine.y; sh->cta_base[lane] = mine.x; }
                 if (lane == 0) sh->cta_base[U] = all;
             }
         }
@@ -876,18 +887,38 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap k_map, co
 // of the others, so a pass costs one memory round trip.  The eight warp results are merged through shared memory.
 constexpr int kCombineThreads = 256;
 template <int D>
-__global__ void __launch_bounds__(kCombineThreads) attn_tc_combine_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kCombineThreads) attn_tc_combine_kernel(const AttnParams p, const int main_grid) {
     constexpr int V = D / 32;   // output columns per lane
     __shared__ float w_m[8], w_l[8];
     __shared__ float w_acc[8][D];
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __shared__ int2 s_info;
     const int R = p.rows, G = p.group, Hkv = p.n_kv_heads;
     const int row = blockIdx.x, tid = threadIdx.x, w = tid >> 5, lane = tid & 31;
     const int h = row % p.n_q_heads, t = (row / p.n_q_heads) % p.q_len, b = row / (p.n_q_heads * p.q_len);
     const int hk = h / G, r = t * G + (h % G);
     __nv_bfloat16 *out = (__nv_bfloat16 *)p.out + (size_t)row * D;
-    const int2 info = reinterpret_cast<const int2 *>(p.counters)[b * Hkv + hk];   // first slot, contributors
+    if (main_grid > 0) {
+        // Unit-aligned split with at most 32 units: which partials belong to this row's unit follows from the lengths
+        // alone.  The lengths are an input of the call, complete before the main kernel let this one be launched, so
+        // the table is worked out here while the main kernel is still running, instead of being read after it.
+        if (w == 0) {
+            const int U = p.batch * Hkv;
+            const int kvl = lane < p.batch ? (p.kv_len ? __ldcg(p.kv_len + lane) : p.max_kv_len) : 0;
+            const int nt = lane < p.batch ? seq_tiles(kvl, p.q_len) : 0;
+            int sum = nt;
+#pragma unroll
+            for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            const int my_tiles = __shfl_sync(0xffffffffu, nt, lane < U ? lane / Hkv : 0);
+            int all;
+            const int2 mine = aligned_split_warp(lane, U, main_grid, lane < U ? my_tiles : 0, (long long)sum * Hkv, all);
+            const int2 pick = make_int2(__shfl_sync(0xffffffffu, mine.x, b * Hkv + hk), __shfl_sync(0xffffffffu, mine.y, b * Hkv + hk));
+            if (lane == 0) s_info = pick;
+        }
+        __syncthreads();
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int2 info = main_grid > 0 ? s_info : reinterpret_cast<const int2 *>(p.counters)[b * Hkv + hk];   // first slot, contributors
     const int n = info.y;
     if (n == 0) {   // a sequence shorter than q_len is skipped: its outputs are defined as zero
         if (tid < D) out[tid] = __float2bfloat16_rn(0.f);
@@ -1068,7 +1099,9 @@ static int32_t launch_tc(const AttnParams &p, int grid, cudaStream_t stream) {
     cfg.gridDim = dim3((unsigned)(p.batch * p.q_len * p.n_q_heads));
     cfg.blockDim = dim3(kCombineThreads);
     cfg.dynamicSmemBytes = 0;
-    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_combine_kernel<D>, p));
+    // unit-aligned split by one warp (see the kernel): the combine kernel derives the slot table itself
+    const int derive = (units <= grid && units <= 32) ? grid : 0;
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc_combine_kernel<D>, p, derive));
     count_launches(1);
     return HIPPO_OK;
 }

@@ -32,8 +32,8 @@ UNIT = "GB/s"
 
 # DRAM traffic of the dominant kernel per launch (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture of
 # the workload named by the key); valid only for the kernel source it was taken on, identified by its hash.
-NCU_TRAFFIC = {"source": "paper_2601_08273_b200/csrc/attn_tc.cu", "sha1_12": "b4d2aec84450",
-               "bytes_per_launch": {"c1_7b_video_6k": 13384448, "c2_long_video_32k": 139715072}}
+NCU_TRAFFIC = {"source": "paper_2601_08273_b200/csrc/attn_tc.cu", "sha1_12": "a4d33593d3d2",
+               "bytes_per_launch": {"c1_7b_video_6k": 13384704, "c2_long_video_32k": 139255552}}
 
 
 def measured_traffic(workload):

@@ -230,3 +230,22 @@ def test_workspace_status_is_clean(hb):
     kv, _, _ = paged_cache(hb, k, k, [100], "bf16")
     hb.hippo_verify_attention(q, kv, dev(np.asarray([100], np.int32)), 100, workspace=ws)
     assert hb.hippo_workspace_status(ws) == hb.HIPPO_OK
+
+
+def test_same_bits_on_repeated_calls(hb):
+    """Full long-video shape: the result does not depend on timing (which CTA finishes first, what ran before)."""
+    cfg = W.CONFIGS[2]
+    q_len = cfg.gamma + 1
+    lens = [W.visual_lengths(cfg)[0] + cfg.n_text + q_len]
+    inp = W.attention_inputs(cfg, "target", lens, q_len)
+    kv, _, _ = paged_cache(hb, inp["k"], inp["v"], lens, "bf16")
+    qd, kvl = dev(inp["q"], "bf16"), dev(np.asarray(lens, np.int32))
+    ws = hb.new_workspace(hb.hippo_attention_workspace_bytes(1, q_len, cfg.tgt_q_heads, cfg.tgt_kv_heads, cfg.tgt_head_dim))
+    outs = []
+    for rep in range(3):
+        if rep:
+            torch.randn(1 << 24, device="cuda").sum().item()      # disturb caches and clocks in between
+        outs.append(host(hb.hippo_verify_attention(qd, kv, kvl, lens[0], workspace=ws)).copy())
+    np.testing.assert_array_equal(outs[0], outs[1])
+    np.testing.assert_array_equal(outs[0], outs[2])
+    assert hb.hippo_workspace_status(ws) == 0

@@ -18,7 +18,9 @@
  *   top-k, gather     - pinned (library sort / exact copy identities).
  *   attention         - pinned (library softmax-attention, closed forms).
  *   attention mass    - pinned (hand-worked case, closed forms, library softmax, invariants).
- *   acceptance        - pinned (losslessness identity by enumeration and by seeded simulation).
+ *   acceptance        - pinned (losslessness identity by enumeration and by seeded simulation); the two
+ *                       margins it reports are pinned by hand-worked cases and by the measured
+ *                       decision boundaries.
  */
 #include <math.h>
 #include <stdint.h>

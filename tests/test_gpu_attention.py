@@ -154,7 +154,9 @@ def sampled_rows(rng, B, q_len, Hq, n):
 
 
 @pytest.mark.parametrize("ci", [1, 2, 4])
-def test_full_size_verify_sampled_rows(hb, ci):
+def test_full_size_verify(hb, ci):
+    """The verification shapes at full size.  Every (token, head) row is compared with the oracle at c1, c2 and at the
+    64k configuration's largest gamma; its other two gammas compare 48 sampled rows."""
     cfg = W.CONFIGS[ci]
     n_v = W.visual_lengths(cfg)[0]
     gammas = W.C4_GAMMA_SWEEP if ci == 4 else (cfg.gamma,)
@@ -163,12 +165,17 @@ def test_full_size_verify_sampled_rows(hb, ci):
         lens = [n_v + cfg.n_text + q_len]
         inp = W.attention_inputs(cfg, "target", lens, q_len)
         got, lse = run_case(hb, hb.hippo_verify_attention, inp["q"], inp["k"], inp["v"], lens, cfg.dtype)
-        rows = sampled_rows(np.random.default_rng(ci), 1, q_len, cfg.tgt_q_heads, 24)
+        assert np.isfinite(got).all()
+        if ci != 4 or g == max(gammas):
+            ref, ref_lse = oracle.attention(inp["q"], inp["k"], inp["v"], lens)
+            assert_close(got, ref, TOL[cfg.dtype], "c%d gamma %d, all rows" % (ci, g))
+            assert_close(lse, ref_lse, 2e-3, "lse")
+            continue
+        rows = sampled_rows(np.random.default_rng(ci), 1, q_len, cfg.tgt_q_heads, 48)
         ref, ref_lse = oracle.attention(inp["q"], inp["k"], inp["v"], lens, rows=rows)
         sel = np.array(rows)
         assert_close(got[sel[:, 0], sel[:, 1], sel[:, 2]], ref, TOL[cfg.dtype], "c%d gamma %d" % (ci, g))
         assert_close(lse[sel[:, 0], sel[:, 1], sel[:, 2]], ref_lse, 2e-3, "lse")
-        assert np.isfinite(got).all()
 
 
 def test_c3_batched_paged_verify_and_draft(hb):
@@ -178,10 +185,8 @@ def test_c3_batched_paged_verify_and_draft(hb):
     lens = [n + cfg.n_text + q_len for n in n_vs]
     inp = W.attention_inputs(cfg, "target", lens, q_len)
     got, _ = run_case(hb, hb.hippo_verify_attention, inp["q"], inp["k"], inp["v"], lens, cfg.dtype, shuffle_seed=33)
-    rows = sampled_rows(np.random.default_rng(3), cfg.batch, q_len, cfg.tgt_q_heads, 32)
-    ref, _ = oracle.attention(inp["q"], inp["k"], inp["v"], lens, rows=rows)
-    sel = np.array(rows)
-    assert_close(got[sel[:, 0], sel[:, 1], sel[:, 2]], ref, TOL[cfg.dtype], "c3 verify")
+    ref, _ = oracle.attention(inp["q"], inp["k"], inp["v"], lens)       # all 8 x 6 x 28 rows
+    assert_close(got, ref, TOL[cfg.dtype], "c3 verify")
     lens_d = [W.keep_count(n, cfg.keep_pct) + cfg.n_text + 1 for n in n_vs]
     inp = W.attention_inputs(cfg, "draft", lens_d, 1)
     got, _ = run_case(hb, hb.hippo_draft_attention, inp["q"], inp["k"], inp["v"], lens_d, cfg.dtype, shuffle_seed=34)

@@ -93,30 +93,25 @@ def test_c3_batched_select(hb):
     inps = [W.select_inputs(cfg, b) for b in range(cfg.batch)]
     ks = [i["k"] for i in inps]
     got = run_select(hb, [i["embeds"] for i in inps], [i["attn_mass"] for i in inps], ks, cfg, "bf16")
-    for b in (0, 3, 7):
+    for b in range(cfg.batch):
         ref_idx, ref_fused, kth = oracle.select_tokens(inps[b]["embeds"], inps[b]["attn_mass"], ks[b], 14, 14)
         check_kept(got[b][0], got[b][1], ref_idx, ref_fused, kth, "c3 seq %d" % b)
 
 
-def test_c4_select_sampled_frames(hb):
-    """Full c4 shape on the GPU; the oracle scores a 6-frame window (frames 99..104) whose inner frames 100..103
-    have complete neighbourhoods, and the GPU's fused scores of those frames must match."""
+def test_c4_select_whole_sequence(hb):
+    """Full c4 shape (65,536 tokens, d = 8192): the oracle scores the whole sequence once; for every kept share of the
+    sweep (50 / 25 / 10 / 5 %) the GPU's fused scores and kept set are compared with it under the near-tie rule."""
     cfg = W.CONFIGS[4]
     inp = W.select_inputs(cfg)
-    ks = [W.keep_count(inp["n_visual"], pct) for pct in W.C4_KEEP_PCT_SWEEP]
-    tpf = cfg.tokens_per_frame
-    E, mass = inp["embeds"], inp["attn_mass"]
-    lo, hi = 99 * tpf, 105 * tpf
-    ref_fused, _, _ = oracle.select_scores(E[lo:hi], mass[lo:hi], cfg.grid_h, cfg.grid_w)
+    E, mass, n = inp["embeds"], inp["attn_mass"], inp["n_visual"]
+    ref_fused, _, _ = oracle.select_scores(E, mass, cfg.grid_h, cfg.grid_w)
     Ed, md = dev(E, "bf16"), dev(mass)
-    for k in ks:
-        kept, fused = hb.hippo_select_tokens(Ed, md, [inp["n_visual"]], [k], cfg.grid_h, cfg.grid_w)
+    for pct in W.C4_KEEP_PCT_SWEEP:
+        k = W.keep_count(n, pct)
+        kept, fused = hb.hippo_select_tokens(Ed, md, [n], [k], cfg.grid_h, cfg.grid_w)
         torch.cuda.synchronize()
-        kept, fused = host(kept), host(fused)
-        np.testing.assert_allclose(fused[lo + tpf:hi - tpf], ref_fused[tpf:-tpf], rtol=0, atol=2e-6)
-        # top-k itself is exact given the GPU's own fp32 scores
-        want = np.sort(np.lexsort((np.arange(fused.size), -fused.astype(np.float64)))[:k])
-        assert kept.tolist() == want.tolist()
+        ref_idx, kth = oracle.topk(ref_fused, k)
+        check_kept(host(kept), host(fused), ref_idx, ref_fused, kth, "c4 keep %d%%" % pct)
 
 
 def test_topk_all_three_key_tiers(hb):
@@ -179,32 +174,42 @@ def test_gather_small_paged(hb, dtype):
     run_gather(hb, cfg, 3, src_lens, keeps, dtype, shuffle=(1, 2))
 
 
-@pytest.mark.parametrize("ci", [1, 2, 3])
-def test_gather_config_shapes(hb, ci):
-    """Keep list = the oracle-independent random kept visual tokens + every text position, as the step does."""
+@pytest.mark.parametrize("ci,keep_pct", [(1, None), (2, None), (3, None), (4, 50), (4, 25), (4, 10), (4, 5)])
+def test_gather_config_shapes(hb, ci, keep_pct):
+    """Keep list = the oracle-independent random kept visual tokens + every text position, as the step does; the
+    64k configuration at each kept share of its sweep."""
     cfg = W.CONFIGS[ci]
+    pct = cfg.keep_pct if keep_pct is None else keep_pct
     rng = np.random.default_rng(ci)
     n_vs = W.visual_lengths(cfg)
     src_lens = [n + cfg.n_text for n in n_vs]
-    keeps = [np.concatenate([np.sort(rng.choice(n, W.keep_count(n, cfg.keep_pct), replace=False)),
+    keeps = [np.concatenate([np.sort(rng.choice(n, W.keep_count(n, pct), replace=False)),
                              np.arange(n, n + cfg.n_text)]) for n in n_vs]
     run_gather(hb, cfg, 2, src_lens, keeps, cfg.dtype, shuffle=(3, 4) if cfg.paged_shuffle else (None, None))
 
 
 # ---- acceptance -----------------------------------------------------------------------------------------------------
 
-def check_accept(hb, inp, what):
+def check_accept(hb, inp, what, forgiven_allowed=0):
+    """Accepted lengths and emitted tokens bit for bit.  A differing sequence is forgiven only when the oracle reports
+    that a uniform sat within 1e-12 (relative) of a decision boundary, and the number forgiven is itself checked:
+    none on the benchmark configurations."""
     n, out = hb.hippo_accept(dev(inp["target_logits"]), dev(inp["draft_logits"]), dev(inp["draft_tokens"]),
                              dev(inp["u_accept"]), dev(inp["u_resample"]))
     torch.cuda.synchronize()
     rn, rout, ma, mc = oracle.accept(inp["target_logits"], inp["draft_logits"], inp["draft_tokens"], inp["u_accept"],
                                      inp["u_resample"])
+    # the margins themselves must be usable: positive and finite wherever a test / a draw was made
+    assert np.all(mc >= 0) and np.all(np.isfinite(mc)), what
+    assert np.all(ma >= 0), what
     n, out = host(n), host(out)
     bad = np.where((n != rn) | (out != rout).any(axis=1))[0]
-    # a mismatch is tolerated only if the oracle reports that a uniform sat within rounding of a decision boundary
+    forgiven = 0
     for b in bad:
         assert min(ma[b], mc[b]) < 1e-12, "%s: sequence %d differs (n %d vs %d, tokens %s vs %s), margins %.3e %.3e" % (
             what, b, n[b], rn[b], out[b], rout[b], ma[b], mc[b])
+        forgiven += 1
+    assert forgiven <= forgiven_allowed, "%s: %d of %d sequences forgiven by the near-boundary rule" % (what, forgiven, len(rn))
     return rn
 
 

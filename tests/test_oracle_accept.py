@@ -224,3 +224,88 @@ def test_greedy_is_the_zero_temperature_limit_of_the_sampling_rule():
     assert n_s.tolist() == n_g.tolist()
     assert out_s.tolist() == out_g.tolist()
     assert len(set(n_g.tolist())) >= 3
+
+
+# ---- the two margins the oracle reports (the GPU parity test reads them to classify a disagreement) -----------------
+
+def margins1(tl, dl, x, ua, ur):
+    n, out, ma, mc = oracle.accept(tl[None], dl[None], np.asarray(x, np.int32)[None], np.asarray(ua, np.float32)[None],
+                                   np.asarray([ur], np.float32))
+    return int(n[0]), out[0].tolist(), float(ma[0]), float(mc[0])
+
+
+def test_margins_on_cases_worked_by_hand():
+    """V = 2 and V = 3 with probabilities that are quarters and halves (logits 0, ln 2, ln 3), so |u Q - P| / P and the
+    distance of u_res Z to the chosen token's CDF edges over Z are numbers written out below."""
+    ln2, ln3 = np.float32(np.log(2.0)), np.float32(np.log(3.0))
+    # P_0 = (1/4, 3/4), Q_0 = (1/2, 1/2), bonus row P_1 = (1/4, 3/4)
+    tl = np.array([[0, ln3], [0, ln3]], np.float32)
+    dl = np.array([[0, 0]], np.float32)
+    # x = 0, u = 1/4: u Q = 1/8 < 1/4 accepted, margin |1/8 - 1/4| / (1/4) = 1/2.  Bonus from P_1 with u_res = 1/2:
+    # CDF edges 1/4, 1 -> token 1, distances 1/4 and 1/2, Z = 1 -> 1/4
+    n, out, ma, mc = margins1(tl, dl, [0], [0.25], 0.5)
+    assert (n, out) == (1, [0, 1])
+    np.testing.assert_allclose([ma, mc], [0.5, 0.25], rtol=0, atol=1e-6)
+    # x = 0, u = 3/4: u Q = 3/8 >= 1/4 rejected, margin (3/8 - 1/4) / (1/4) = 1/2.  Residual (0, 1/4), Z = 1/4,
+    # u_res = 3/8 -> target 3/32 in token 1's interval (0, 1/4]: distances 3/32 and 5/32 -> (3/32) / (1/4) = 3/8
+    n, out, ma, mc = margins1(tl, dl, [0], [0.75], 0.375)
+    assert (n, out) == (0, [1, -1])
+    np.testing.assert_allclose([ma, mc], [0.5, 0.375], rtol=0, atol=1e-6)
+    # x = 1: P/Q = 3/2, always accepted; u = 1/2: |1/4 - 3/4| / (3/4) = 2/3.  Bonus with u_res = 1/8: token 0,
+    # interval [0, 1/4): distances 1/8 and 1/8 -> 1/8
+    n, out, ma, mc = margins1(tl, dl, [1], [0.5], 0.125)
+    assert (n, out) == (1, [1, 0])
+    np.testing.assert_allclose([ma, mc], [2.0 / 3.0, 0.125], rtol=0, atol=1e-6)
+    # V = 3, two draft rows: the accept margin is the minimum over the tests made.  P = (1/2, 1/4, 1/4) in every row,
+    # Q = (1/4, 1/4, 1/2).  Row 0: x = 2, u = 1/4: u Q = 1/8 < 1/4 accepted, margin 1/2.  Row 1: x = 2, u = 7/16:
+    # u Q = 7/32 < 1/4 accepted, margin 1/8.  Bonus from P with u_res = 5/8: CDF 1/2, 3/4, 1 -> token 1,
+    # distances 1/8 and 1/8 -> 1/8
+    tl3 = np.array([[ln2, 0, 0]] * 3, np.float32)
+    dl3 = np.array([[0, 0, ln2]] * 2, np.float32)
+    n, out, ma, mc = margins1(tl3, dl3, [2, 2], [0.25, 0.4375], 0.625)
+    assert (n, out) == (2, [2, 2, 1])
+    np.testing.assert_allclose([ma, mc], [0.125, 0.125], rtol=0, atol=1e-6)
+    # row 1 rejected instead (u = 3/4: u Q = 3/8 >= 1/4, margin 1/2): the minimum stays row 0's 1/2; the second row's
+    # test is the last one made.  Residual (1/4, 0, 0), Z = 1/4, u_res = 1/2: token 0, distances 1/8 and 1/8 -> 1/2
+    n, out, ma, mc = margins1(tl3, dl3, [2, 2], [0.25, 0.75], 0.5)
+    assert (n, out) == (1, [2, 0, -1])
+    np.testing.assert_allclose([ma, mc], [0.5, 0.5], rtol=0, atol=1e-6)
+    # a rejection at row 0 makes no test at row 1: a uniform there that sits almost on its boundary must not show
+    n, out, ma, mc = margins1(tl3, dl3, [2, 2], [0.75, 0.5], 0.5)
+    assert n == 0
+    np.testing.assert_allclose(ma, 0.5, rtol=0, atol=1e-6)
+
+
+def test_margins_vanish_at_the_measured_decision_boundaries():
+    """The accept margin at u is |u - u*| / u* for the boundary u* = P/Q that the oracle's own decisions flip at (located
+    by bisection over fp32 uniforms), and the CDF margin is the distance of u_res to the nearer measured edge of the
+    emitted token's interval: both go to zero there, and nowhere else."""
+    rng = np.random.default_rng(21)
+    V = 6
+    tl = (rng.standard_normal((2, V)) * 1.5).astype(np.float32)
+    dl = (rng.standard_normal((1, V)) * 1.5).astype(np.float32)
+    P, Q = softmax(tl[0].astype(np.float64)), softmax(dl[0].astype(np.float64))
+    x = int(np.argmax(Q / P))                     # a token the draft over-weights: P/Q < 1, the boundary is inside (0, 1)
+    u_star = accept_measure(tl, dl, x)
+    np.testing.assert_allclose(u_star, P[x] / Q[x], atol=1e-6)
+    for u in (0.1 * u_star, 0.5 * u_star, 0.999 * u_star, 1.001 * u_star, min(0.999, 1.5 * u_star)):
+        u32 = float(np.float32(u))
+        _, _, ma, _ = margins1(tl, dl, [x], [u32], 0.5)
+        np.testing.assert_allclose(ma, abs(u32 - u_star) / u_star, atol=2e-6)
+    below, above = np.nextafter(np.float32(u_star), np.float32(0)), np.nextafter(np.float32(u_star), np.float32(1))
+    assert margins1(tl, dl, [x], [below], 0.5)[2] < 1e-6 and margins1(tl, dl, [x], [above], 0.5)[2] < 1e-6
+    # CDF margin after a rejection: edges of the residual distribution measured from the emitted tokens
+    w = np.maximum(0.0, P - Q)
+    edges = np.concatenate([[0.0], np.cumsum(w) / w.sum()])
+    for u_res in (0.03, 0.2, 0.41, 0.77, 0.96):
+        u32 = float(np.float32(u_res))
+        n, out, _, mc = margins1(tl, dl, [x], [np.nextafter(np.float32(1), np.float32(0))], u32)
+        assert n == 0
+        t = out[0]
+        assert edges[t] <= u32 < edges[t + 1]
+        np.testing.assert_allclose(mc, min(u32 - edges[t], edges[t + 1] - u32), atol=1e-7)
+    # approaching an interior edge from both sides
+    e = float(edges[np.flatnonzero(w > 0)[0] + 1])
+    if 0.0 < e < 1.0:
+        for u_res in (np.float32(e) - np.float32(1e-6), np.float32(e) + np.float32(1e-6)):
+            assert margins1(tl, dl, [x], [0.9999999], float(u_res))[3] < 3e-6

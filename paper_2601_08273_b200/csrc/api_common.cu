@@ -1,5 +1,6 @@
 // Status strings, per-thread error text and workspace header helpers.
 #include <stdarg.h>
+#include <stddef.h>
 #include <string.h>
 
 #include <atomic>
@@ -64,6 +65,17 @@ int32_t hippo_workspace_status(const void *workspace, void *stream) {
     HIPPO_CUDA_TRY(cudaMemcpyAsync(&h, workspace, sizeof(int32_t) * 2, cudaMemcpyDeviceToHost, s));
     HIPPO_CUDA_TRY(cudaStreamSynchronize(s));
     if (h.status != 0) return hippo::fail(h.status, "device-side wait gave up (site %d)", h.where);
+    return HIPPO_OK;
+}
+
+int32_t hippo_workspace_set_wait_limit(void *workspace, int64_t limit_ns, void *stream) {
+    if (!workspace) return hippo::fail(HIPPO_ERR_INVALID_ARG, "hippo_workspace_set_wait_limit: null workspace");
+    if (limit_ns < 0) return hippo::fail(HIPPO_ERR_INVALID_ARG, "hippo_workspace_set_wait_limit: negative limit");
+    cudaStream_t s = (cudaStream_t)stream;
+    long long v = (long long)limit_ns;
+    HIPPO_CUDA_TRY(cudaMemcpyAsync((char *)workspace + offsetof(hippo::WsHeader, wait_limit_ns), &v, sizeof(v),
+                                   cudaMemcpyHostToDevice, s));
+    HIPPO_CUDA_TRY(cudaStreamSynchronize(s));   // `v` lives on this stack frame
     return HIPPO_OK;
 }
 

@@ -72,29 +72,36 @@ struct MassParams {
 
 struct MassShared {
     unsigned long long full[kMassSlots], empty[kMassSlots], res_full[2], res_free[2], s_full[2], s_free[2], drain;
+    long long wait_limit;   // the header's wait limit (0: the built-in one), read once
     uint32_t tmem_base;
     volatile int abort;
 };
 
-__device__ __noinline__ bool mass_wait_slow(MassShared *sh, WsHeader *hdr, uint32_t b, uint32_t parity, int site) {
+// Polling part of a bounded wait.  The limit is kMassWaitLimitNs unless the workspace header carries another one (a
+// debugging aid, read once per CTA into shared memory): then the waits poll without suspending and look at the clock
+// after every poll.  A drain wait guards the exit of the CTA (loads in flight, tensor-core work in flight): it keeps the
+// built-in limit and does not give up because another wait did.
+__device__ __noinline__ bool mass_wait_slow(MassShared *sh, WsHeader *hdr, uint32_t b, uint32_t parity, int site, bool draining) {
     const unsigned long long t0 = global_ns();
+    const long long user = draining ? 0 : sh->wait_limit;
+    const unsigned long long limit = user > 0 ? (unsigned long long)user : kMassWaitLimitNs;
     for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(b, parity)) return true;
-        if ((i & 31) == 0) {
-            if (sh->abort) return false;
-            if (global_ns() - t0 > kMassWaitLimitNs) {
+        if (user > 0 ? mbar_test_wait(b, parity) : mbar_try_wait(b, parity)) return true;
+        if (user > 0 || (i & 31) == 0) {
+            if (!draining && sh->abort) return false;
+            if (global_ns() - t0 > limit) {
                 sh->abort = 1;
-                atomicExch(&hdr->status, (int)HIPPO_ERR_TIMEOUT);
-                hdr->where = 100 + site;
+                if (atomicCAS(&hdr->status, 0, (int)HIPPO_ERR_TIMEOUT) == 0) hdr->where = 100 + site;
                 return false;
             }
         }
     }
 }
-__device__ __forceinline__ bool mass_wait(MassShared *sh, WsHeader *hdr, unsigned long long *bar, uint32_t parity, int site) {
+__device__ __forceinline__ bool mass_wait(MassShared *sh, WsHeader *hdr, unsigned long long *bar, uint32_t parity, int site,
+                                          bool draining = false) {
     const uint32_t b = smem_u32(bar);
-    if (mbar_try_wait(b, parity)) return true;
-    return mass_wait_slow(sh, hdr, b, parity, site);
+    if ((!draining && sh->wait_limit > 0) ? mbar_test_wait(b, parity) : mbar_try_wait(b, parity)) return true;
+    return mass_wait_slow(sh, hdr, b, parity, site, draining);
 }
 
 // PASS 0: row statistics (resident Q block, streamed key tiles).  PASS 1: column sums (resident key tile, streamed Q blocks).
@@ -153,7 +160,7 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
     else if (tid >= 52 && tid < 54) mbar_init(smem_u32(&sh->s_full[tid - 52]), 1);
     else if (tid >= 54 && tid < 56) mbar_init(smem_u32(&sh->s_free[tid - 54]), kMassConsumers);
     else if (tid == 56) mbar_init(smem_u32(&sh->drain), 1);
-    else if (tid == 57) sh->abort = 0;
+    else if (tid == 57) { sh->abort = 0; sh->wait_limit = p.header->wait_limit_ns; }
     if (tid == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
@@ -216,10 +223,10 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
             const int back = issued < (uint32_t)kSlots ? (int)issued : kSlots;
             for (int k = 0; k < back; ++k) {
                 if (rp.slot == 0) { rp.slot = kSlots - 1; rp.phase ^= 1; } else --rp.slot;
-                mass_wait(sh, hdr, &sh->full[rp.slot], rp.phase, 3);
+                mass_wait(sh, hdr, &sh->full[rp.slot], rp.phase, 3, true);
             }
             for (uint32_t k = res_issued > (uint32_t)kRes ? res_issued - kRes : 0; k < res_issued; ++k)
-                mass_wait(sh, hdr, &sh->res_full[k % kRes], (k / kRes) & 1, 4);
+                mass_wait(sh, hdr, &sh->res_full[k % kRes], (k / kRes) & 1, 4, true);
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
@@ -255,7 +262,7 @@ mass_tc_kernel(const MassParams p, const __grid_constant__ CUtensorMap k_map, co
             }
             // all tensor-core work of this CTA must be complete before tensor memory is released
             tc_commit(smem_u32(&sh->drain));
-            mass_wait(sh, hdr, &sh->drain, 0, 8);
+            mass_wait(sh, hdr, &sh->drain, 0, 8, true);
         }
     } else {
         // ================= consumers =================

@@ -19,9 +19,10 @@ constexpr int kExtraSlots = 4 * kNumSMs;     // partial-result slots beyond one 
 
 // First bytes of every workspace.
 struct WsHeader {
-    int32_t status;      // 0, or HIPPO_ERR_TIMEOUT once a bounded wait gave up
-    int32_t where;       // code of the wait that gave up (debugging aid)
-    int32_t pad[62];
+    int32_t status;          // 0, or HIPPO_ERR_TIMEOUT once a bounded wait gave up
+    int32_t where;           // code of the wait that gave up (debugging aid)
+    long long wait_limit_ns; // 0: the built-in limit; else the limit of the bounded waits (hippo_workspace_set_wait_limit)
+    int32_t pad[60];
 };
 static_assert(sizeof(WsHeader) == kWsHeaderBytes, "header size");
 
@@ -85,6 +86,7 @@ struct AttnParams {
     const void *v_pages;
     const int32_t *page_table;   // may be null: identity
     const int32_t *kv_len;
+    const int32_t *kv_len_host;  // may be null: host copy of kv_len, used only to plan the launch
     WsHeader *header;
     int32_t *counters;
     float *partials;             // n_slots x slot_float_count(rows, D) floats
@@ -106,8 +108,16 @@ __device__ __forceinline__ int page_of(const int32_t *page_table, int max_pages_
 // entry points implemented per translation unit
 int32_t launch_attn_generic(const AttnParams &p, int dtype, cudaStream_t stream);
 int32_t launch_attn_combine(const AttnParams &p, int dtype, int n_splits, cudaStream_t stream);
-int32_t launch_attn_tc(const AttnParams &p, bool draft_policy, cudaStream_t stream);
+int32_t launch_attn_tc(const AttnParams &p, cudaStream_t stream);
 bool attn_tc_supported(const AttnParams &p, int dtype);
+// several layers in one launch: header | per-unit slot table | done[layers][units], merged[layers] | slot sets
+struct AttnLayersWsLayout {
+    size_t counters_off, done_off, done_bytes, partials_off, slot_floats, slots_per_set, total;
+};
+AttnLayersWsLayout attn_layers_ws_layout(int n_layers, int batch, int q_len, int n_q_heads, int n_kv_heads, int head_dim);
+bool attn_tc_layers_supported(const AttnParams &p, int dtype);
+int32_t launch_attn_tc_layers(const AttnParams &p, int n_layers, const void *const *q, const hippo_kv_cache_t *kv,
+                              void *const *out, float *const *lse, void *workspace, cudaStream_t stream);
 int32_t launch_attn_small(const AttnParams &p, cudaStream_t stream);
 bool attn_small_supported(const AttnParams &p, int dtype);
 

@@ -23,7 +23,7 @@ def test_library_exports_every_declared_symbol():
             "hippo_accept"} <= set(names)
     for n in names:
         assert hasattr(binding.lib, n), n
-    assert binding.hippo_version() == 100
+    assert binding.hippo_version() == 101
     assert binding.lib.hippo_status_string(-5).decode() == "device-side wait timed out"
 
 
@@ -36,13 +36,14 @@ def test_argument_validation_happens_before_any_launch():
     assert lib.hippo_accept(1, 1, 10, 256, 256, 256, 256, 256, 7, 256, 256, 256, 1 << 20, None) == hb.HIPPO_ERR_UNIMPLEMENTED   # unknown mode
     assert lib.hippo_accept(1, 1, 10, 256, 256, 256, 256, 256, 0, 256, 256, 256, 16, None) == hb.HIPPO_ERR_WORKSPACE_TOO_SMALL
     kv = hb.KVCacheStruct(ctypes.sizeof(hb.KVCacheStruct), hb.HIPPO_DTYPE_BF16, 2, 64, 10, 4, 1024, 2048, None)
-    args = lambda **o: [o.get("B", 1), o.get("q_len", 1), o.get("hq", 14), 256, ctypes.byref(kv), 256,
+    args = lambda **o: [o.get("B", 1), o.get("q_len", 1), o.get("hq", 14), 256, ctypes.byref(kv), 256, o.get("host_len"),
                         o.get("max_kv", 200), 0.0, 0, 256, None, o.get("ws", 256), o.get("ws_bytes", 1 << 30), None]
     assert lib.hippo_draft_attention(*args(hq=15)) == hb.HIPPO_ERR_INVALID_ARG          # 15 % 2 != 0
     assert lib.hippo_draft_attention(*args(max_kv=257)) == hb.HIPPO_ERR_INVALID_ARG      # > 4 pages
     assert lib.hippo_draft_attention(*args(ws_bytes=1000)) == hb.HIPPO_ERR_WORKSPACE_TOO_SMALL
     assert lib.hippo_draft_attention(*args(q_len=40)) == hb.HIPPO_ERR_UNSUPPORTED_SHAPE  # 40*7 packed rows
     assert lib.hippo_draft_attention(*args(B=3)) == hb.HIPPO_ERR_INVALID_ARG             # identity mapping needs 12 pages
+    assert lib.hippo_draft_attention(*args(host_len=(ctypes.c_int32 * 1)(201))) == hb.HIPPO_ERR_INVALID_ARG   # host length > max_kv_len
     kv.struct_size = 8
     assert lib.hippo_verify_attention(*args()) == hb.HIPPO_ERR_INVALID_ARG
     n_visual = (ctypes.c_int32 * 1)(100)

@@ -150,3 +150,29 @@ def test_reproducible_bits(hb):
     torch.randn(1 << 22, device="cuda").sum().item()
     b = gpu_mass(hb, [inp["q_txt"]], [inp["k_vid"]], nv, cfg.dtype)
     np.testing.assert_array_equal(a, b)
+
+
+def test_bounded_wait_runs_out_and_the_workspace_recovers(hb):
+    """The same exercise as for the attention kernels: a 200 ns wait limit makes the first wait of the tensor-core
+    mass kernel give up while every load still lands; the kernel returns, the status word says so, a reset clears it
+    and the next call matches the oracle."""
+    rng = np.random.default_rng(8)
+    B, L, Hq, Hkv, D, nv = 1, 16, 8, 2, 128, [1500]
+    q = W.round_to_storage(rng.standard_normal((B, L, Hq, D)).astype(np.float32), "bf16")
+    k = W.round_to_storage(rng.standard_normal((B, nv[0], Hkv, D)).astype(np.float32), "bf16")
+    kv, _, _ = paged_cache(hb, k, k, nv, "bf16")
+    qd = dev(q, "bf16")
+    ws = hb.new_workspace(hb.hippo_attention_mass_workspace_bytes(nv, L, Hq, Hkv, D, hb.HIPPO_DTYPE_BF16))
+    mass = torch.zeros(nv[0], dtype=torch.float32, device="cuda")
+    w = 1.0 / (Hq * L)
+    hb.hippo_workspace_set_wait_limit(ws, 200)
+    hb.hippo_attention_mass(qd, kv, nv, w, mass, workspace=ws)
+    assert hb.hippo_workspace_status(ws) == hb.HIPPO_ERR_TIMEOUT
+    hb.hippo_workspace_reset(ws)
+    assert hb.hippo_workspace_status(ws) == hb.HIPPO_OK
+    mass.zero_()
+    hb.hippo_attention_mass(qd, kv, nv, w, mass, workspace=ws)
+    assert hb.hippo_workspace_status(ws) == hb.HIPPO_OK
+    ref = oracle.attention_mass(q[None], k[None], nv)[0][:nv[0]]
+    got = host(mass)
+    assert np.all(np.abs(got - ref) <= RTOL["bf16"] * ref + 1e-12)

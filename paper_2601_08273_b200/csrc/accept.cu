@@ -187,10 +187,14 @@ __device__ RowInfo decide_rows(const AcceptParams &p, int b, double *rowstat /* 
             bool accept = true;
             if (j < p.gamma) {
                 const int rq = p.gamma + 1 + j, tok = x[j];
-                const double P = exp((double)logit_row(p, b, j)[tok] - rowstat[2 * j]) / rowstat[2 * j + 1];
-                const double Q = exp((double)logit_row(p, b, rq)[tok] - rowstat[2 * rq]) / rowstat[2 * rq + 1];
-                const double u = (double)p.ua[(size_t)b * p.gamma + j];
-                accept = u * Q < P;
+                // a token id outside the vocabulary (a fault upstream) is never looked up: it counts as rejected
+                accept = false;
+                if ((unsigned)tok < (unsigned)p.V) {
+                    const double P = exp((double)logit_row(p, b, j)[tok] - rowstat[2 * j]) / rowstat[2 * j + 1];
+                    const double Q = exp((double)logit_row(p, b, rq)[tok] - rowstat[2 * rq]) / rowstat[2 * rq + 1];
+                    const double u = (double)p.ua[(size_t)b * p.gamma + j];
+                    accept = u * Q < P;
+                }
             }
             const unsigned rejected = __ballot_sync(0xffffffffu, !accept);
             if (rejected) { n = j0 + __ffs(rejected) - 1; break; }
@@ -531,10 +535,12 @@ extern "C" int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vo
                                         void *stream) {
     using namespace hippo;
     if (batch <= 0 || gamma < 0 || vocab <= 0) return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: bad sizes");
-    if (mode != HIPPO_ACCEPT_SAMPLE) return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept_noalloc: mode %d", mode);
-    if (!target_logits || !u_resample || !n_accepted || !out_tokens)
+    if (mode != HIPPO_ACCEPT_SAMPLE && mode != HIPPO_ACCEPT_GREEDY)
+        return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept_noalloc: mode %d", mode);
+    const bool greedy = mode == HIPPO_ACCEPT_GREEDY;
+    if (!target_logits || !n_accepted || !out_tokens || (!greedy && !u_resample))
         return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: null pointer");
-    if (gamma > 0 && (!draft_logits || !draft_tokens || !u_accept))
+    if (gamma > 0 && (!draft_tokens || (!greedy && (!draft_logits || !u_accept))))
         return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: null draft arrays with gamma > 0");
     if (gamma > 64 || batch > 65535) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_accept_noalloc: gamma > 64 or batch > 65535");
     const AcceptWs w = accept_ws(batch, gamma, vocab);
@@ -558,5 +564,5 @@ extern "C" int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vo
     p.tscan = (double *)((char *)scratch + w.tscan_off);
     p.B = batch; p.gamma = gamma; p.V = vocab; p.n_chunks = w.n_chunks;
     cudaStream_t s = (cudaStream_t)stream;
-    return launch_accept(p, s);
+    return greedy ? launch_accept_greedy(p, s) : launch_accept(p, s);
 }

@@ -1,8 +1,8 @@
 // hippo_gather_kv: compacts the kept rows of the draft model's KV cache, all layers in one launch.
 //
-// "One-time pruning of the draft model's KV cache during the prefill stage" (Limitations (i)): after selection the
-// draft keeps only the chosen visual tokens plus the always-kept positions.  A pure copy, bound by HBM bandwidth:
-// per kept token and layer 2 * n_kv_heads * head_dim elements are read and written once.
+// The draft model's cache is pruned once, during prefill (Limitations (i)): after selection the draft keeps only the
+// chosen visual tokens plus the always-kept positions.  A pure copy, bound by HBM bandwidth: per kept token and layer
+// 2 * n_kv_heads * head_dim elements are read and written once.
 //
 // One work item is a 16-byte piece of one kept row: (chunk within row, destination token, head).  Its offsets inside a
 // (layer, K|V) plane are the same for every plane - the page tables are shared by all layers - so a thread resolves
@@ -11,6 +11,12 @@
 // fill the machine.  Items are ordered so that consecutive threads write consecutive addresses of one destination
 // (page, head) block; reads are whole rows of head_dim elements (128 B for head_dim 64 bf16) scattered over the
 // source pages.
+//
+// Indices come from device memory (a selector's output, an engine's page tables), so every address formed from them is
+// checked first: a source position beyond the sequence's page capacity, a destination position beyond the destination's,
+// or a page id outside its pool skips the item and raises the caller's flag word instead of touching memory.
+#include <initializer_list>
+
 #include "common.cuh"
 
 namespace hippo {
@@ -19,8 +25,10 @@ struct GatherParams {
     const char *src_k, *src_v;
     char *dst_k, *dst_v;
     const int32_t *src_table, *dst_table, *keep_idx, *keep_offsets;
+    int32_t *bad_index;          // may be null: set to 1 when an item was skipped
     size_t src_layer_stride, dst_layer_stride;
     int n_layers, batch, total_keep, n_kv_heads, row_chunks, src_mpps, dst_mpps, planes_per_group;
+    int src_pages, dst_pages;    // pool sizes
 };
 
 constexpr int kGatherThreads = 256;
@@ -40,8 +48,19 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kv_kernel(const GatherP
     }
     const int src_tok = __ldg(p.keep_idx + i);
     const int dst_tok = i - __ldg(p.keep_offsets + lo);
-    const int sp = page_of(p.src_table, p.src_mpps, lo, src_tok / kPageSize);
-    const int dp = page_of(p.dst_table, p.dst_mpps, lo, dst_tok / kPageSize);
+    // positions must lie inside the page-table rows before the tables are read, page ids inside the pools before
+    // the pools are
+    bool ok = src_tok >= 0 && src_tok < p.src_mpps * kPageSize && dst_tok >= 0 && dst_tok < p.dst_mpps * kPageSize;
+    int sp = 0, dp = 0;
+    if (ok) {
+        sp = page_of(p.src_table, p.src_mpps, lo, src_tok / kPageSize);
+        dp = page_of(p.dst_table, p.dst_mpps, lo, dst_tok / kPageSize);
+        ok = sp >= 0 && sp < p.src_pages && dp >= 0 && dp < p.dst_pages;
+    }
+    if (!ok) {
+        if (p.bad_index) *p.bad_index = 1;
+        return;
+    }
     const size_t row_bytes = (size_t)p.row_chunks * 16;
     const size_t so = (((size_t)sp * p.n_kv_heads + h) * kPageSize + (src_tok % kPageSize)) * row_bytes + c * 16u;
     const size_t dof = (((size_t)dp * p.n_kv_heads + h) * kPageSize + (dst_tok % kPageSize)) * row_bytes + c * 16u;
@@ -78,7 +97,7 @@ static int32_t check(const hippo_kv_cache_t *kv, const char *name) {
 extern "C" int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src, size_t src_layer_stride_bytes,
                                    const hippo_kv_cache_t *dst, size_t dst_layer_stride_bytes, int32_t batch,
                                    const int32_t *keep_idx, const int32_t *keep_offsets, int32_t total_keep,
-                                   void *stream) {
+                                   int32_t *bad_index, void *stream) {
     using namespace hippo;
     int32_t rc = check(src, "src");
     if (rc != HIPPO_OK) return rc;
@@ -94,6 +113,12 @@ extern "C" int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src
     if (row_bytes % 16) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "hippo_gather_kv: head_dim*elem_size must be a multiple of 16 bytes");
     if ((src_layer_stride_bytes | dst_layer_stride_bytes) & 127)
         return fail(HIPPO_ERR_INVALID_ARG, "hippo_gather_kv: layer strides must be multiples of 128 bytes");
+    if ((long long)total_keep > (long long)batch * dst->max_pages_per_seq * kPageSize)
+        return fail(HIPPO_ERR_INVALID_ARG, "hippo_gather_kv: total_keep %d exceeds the destination's capacity (%d sequences x %d pages)",
+                    total_keep, batch, dst->max_pages_per_seq);
+    for (const hippo_kv_cache_t *kv : {src, dst})
+        if (!kv->page_table && (long long)batch * kv->max_pages_per_seq > kv->n_pages)
+            return fail(HIPPO_ERR_INVALID_ARG, "hippo_gather_kv: identity page mapping needs batch*max_pages_per_seq <= n_pages");
     if (total_keep == 0) return HIPPO_OK;
     if (!keep_idx || !keep_offsets) return fail(HIPPO_ERR_INVALID_ARG, "hippo_gather_kv: null index arrays");
 
@@ -101,7 +126,8 @@ extern "C" int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src
     p.src_k = (const char *)src->k_pages; p.src_v = (const char *)src->v_pages;
     p.dst_k = (char *)dst->k_pages; p.dst_v = (char *)dst->v_pages;
     p.src_table = src->page_table; p.dst_table = dst->page_table;
-    p.keep_idx = keep_idx; p.keep_offsets = keep_offsets;
+    p.keep_idx = keep_idx; p.keep_offsets = keep_offsets; p.bad_index = bad_index;
+    p.src_pages = src->n_pages; p.dst_pages = dst->n_pages;
     p.src_layer_stride = src_layer_stride_bytes; p.dst_layer_stride = dst_layer_stride_bytes;
     p.n_layers = n_layers; p.batch = batch; p.total_keep = total_keep; p.n_kv_heads = src->n_kv_heads;
     p.row_chunks = (int)(row_bytes / 16); p.src_mpps = src->max_pages_per_seq; p.dst_mpps = dst->max_pages_per_seq;

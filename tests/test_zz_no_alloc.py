@@ -41,6 +41,34 @@ def test_noalloc_matches_hippo_accept_twice_in_a_row():
         assert (host(got_n) >= 0).all() and (host(got_n) <= g1 - 1).all()
 
 
+def test_noalloc_calls_back_to_back_on_one_stream():
+    """Three different problems enqueued on one stream with no synchronisation in between - sampling, no draft tokens at
+    all (gamma = 0), greedy - all sharing the built-in array: stream order alone must keep them apart.  Checked after a
+    single synchronisation against hippo_accept with its own workspaces."""
+    from paper_2601_08273_b200 import binding as hb
+    cfg = W.CONFIGS[1]
+    names = ("target_logits", "draft_logits", "draft_tokens", "u_accept", "u_resample")
+    a = W.accept_inputs(cfg, batch=4, corr_eps=0.2, sub=21)
+    b = W.accept_inputs(cfg, batch=3, gamma=0, vocab=9001, sub=22)
+    c = W.accept_inputs(cfg, batch=5, gamma=4, vocab=50001, corr_eps=0.0, sub=23)
+    c["draft_tokens"] = c["target_logits"][:, :4].argmax(axis=-1).astype(np.int32)
+    c["draft_tokens"][2, 1] += 1
+    dev_in = [[dev(x[k]) for k in names] for x in (a, b, c)]
+    modes = (hb.HIPPO_ACCEPT_SAMPLE, hb.HIPPO_ACCEPT_SAMPLE, hb.HIPPO_ACCEPT_GREEDY)
+    want = [hb.hippo_accept(*args, mode=m) for args, m in zip(dev_in, modes)]
+    got = [(torch.full((x["target_logits"].shape[0],), -7, dtype=torch.int32, device="cuda"),
+            torch.full(x["target_logits"].shape[:2], -7, dtype=torch.int32, device="cuda")) for x in (a, b, c)]
+    torch.cuda.synchronize()
+    for rep in range(2):
+        for args, m, (gn, gt) in zip(dev_in, modes, got):
+            hb.hippo_accept_noalloc(*args, gn, gt, mode=m)
+    torch.cuda.synchronize()
+    for (wn, wt), (gn, gt) in zip(want, got):
+        np.testing.assert_array_equal(host(gn), host(wn))
+        np.testing.assert_array_equal(host(gt), host(wt))
+    assert host(got[2][0]).tolist() == [4, 4, 1, 4, 4]
+
+
 def test_noalloc_refuses_sizes_beyond_its_array():
     from paper_2601_08273_b200 import binding as hb
     B, g, V = 64, 8, 152064

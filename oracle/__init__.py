@@ -93,6 +93,22 @@ def select_tokens(embeds, attn_mass, k: int, grid_h: int, grid_w: int, crop_h: i
     return idx, fused, kth
 
 
+POLICY_HOLISTIC, POLICY_UNIFORM_PER_FRAME, POLICY_RANDOM, POLICY_FRAME = 0, 1, 2, 3
+
+
+def select_policy(policy: int, score, k: int, tokens_per_frame: int):
+    """The kept indices (ascending) under one of the selection rules; `score` is the fused score (policies 0, 1), the
+    caller's random keys (policy 2) or ignored (policy 3).  Returns (kept int32[k], per-frame budget int32[F])."""
+    s = np.ascontiguousarray(score, dtype=np.float64)
+    n = s.shape[0]
+    idx = np.empty(k, dtype=np.int32)
+    budget = np.zeros((n + tokens_per_frame - 1) // tokens_per_frame, dtype=np.int32)
+    rc = _load().oracle_select_policy(policy, n, tokens_per_frame, _p(s), k, _p(idx), _p(budget))
+    if rc != 0:
+        raise ValueError("oracle_select_policy rc=%d" % rc)
+    return idx, budget
+
+
 def gather_kv(src, keep) -> np.ndarray:
     """src [n_layers][n_src][...row...] (any dtype) -> dst [n_layers][len(keep)][...row...]."""
     s = np.ascontiguousarray(src)

@@ -225,6 +225,72 @@ int oracle_topk(int n, const double *score, int k, int32_t *kept_idx, double *kt
 }
 
 /* ------------------------------------------------------------------------------------------------
+ * Other selection rules, for comparison with the holistic rule above.  The paper names them without
+ * spelling them out: uniform pruning across all frames (related work, the attention-guided selection
+ * of an earlier video speculative-decoding method), randomly sampled tokens and whole frames dropped at
+ * regular temporal intervals (Section 6, exploration of pruning criteria).  The readings taken:
+ *   policy 0  holistic    the k best over the whole sequence (oracle_topk).
+ *   policy 1  per frame   every frame gets the same budget: floor(k / F) tokens, the first k mod F frames
+ *                         one more; a frame that holds fewer tokens than its budget (a partial last
+ *                         frame) keeps them all and the shortfall goes, one token at a time in frame
+ *                         order, to the frames that still have room.  Inside a frame the best tokens by
+ *                         (score descending, index ascending).
+ *   policy 2  random      the k best by a caller-supplied key per token (the caller draws the keys): the
+ *                         same rule as policy 0 with the keys as scores.
+ *   policy 3  frames      whole frames at a regular stride: with m = ceil(k / T) frames to keep out of the
+ *                         Fc complete frames (T tokens each), frame floor(i * Fc / m) for i = 0..m-1; when k
+ *                         is not a multiple of T the last kept frame gives only its first cells.  If k
+ *                         reaches Fc * T (or there is no complete frame) the complete frames are all kept
+ *                         and the rest comes from the first cells of the partial frame.
+ * score: [n] (ignored by policy 3).  frame_budget (may be NULL): [F] tokens kept per frame, for policy 1.
+ * ---------------------------------------------------------------------------------------------- */
+int oracle_select_policy(int policy, int n, int tokens_per_frame, const double *score, int k, int32_t *kept_idx,
+                         int32_t *frame_budget) {
+    if (n <= 0 || tokens_per_frame <= 0 || k < 0 || k > n) return -1;
+    int T = tokens_per_frame, F = (n + T - 1) / T;
+    if (policy == 0 || policy == 2) return oracle_topk(n, score, k, kept_idx, NULL);
+    if (policy == 1) {
+        int *budget = (int *)malloc((size_t)F * sizeof(int));
+        if (!budget) return -2;
+        int given = 0;
+        for (int f = 0; f < F; ++f) {
+            int want = k / F + (f < k % F ? 1 : 0), have = frame_tokens(n, T, f);
+            budget[f] = want < have ? want : have;
+            given += budget[f];
+        }
+        while (given < k)
+            for (int f = 0; f < F && given < k; ++f)
+                if (budget[f] < frame_tokens(n, T, f)) { ++budget[f]; ++given; }
+        int out = 0;
+        for (int f = 0; f < F; ++f) {
+            int have = frame_tokens(n, T, f);
+            int rc = oracle_topk(have, score + (size_t)f * T, budget[f], kept_idx + out, NULL);
+            if (rc != 0) { free(budget); return rc; }
+            for (int i = 0; i < budget[f]; ++i) kept_idx[out + i] += f * T;
+            out += budget[f];
+            if (frame_budget) frame_budget[f] = budget[f];
+        }
+        free(budget);
+        return 0;
+    }
+    if (policy == 3) {
+        int Fc = n / T, out = 0;
+        if (Fc == 0 || (long)k >= (long)Fc * T) {
+            for (int i = 0; i < k; ++i) kept_idx[i] = i;      /* all complete frames, then the first cells of the rest */
+            return 0;
+        }
+        int m = (k + T - 1) / T;
+        for (int i = 0; i < m; ++i) {
+            int f = (int)((long)i * Fc / m);
+            int take = k - out < T ? k - out : T;
+            for (int c = 0; c < take; ++c) kept_idx[out++] = f * T + c;
+        }
+        return 0;
+    }
+    return -1;
+}
+
+/* ------------------------------------------------------------------------------------------------
  * Gather: "one-time pruning of the draft model's KV cache" (Limitations (i)); removing the pruned
  * video features (experimental set-up).  dst[l][i][h][:] = src[l][keep[i]][h][:].
  * src [n_layers][n_src][row], dst [n_layers][n_keep][row], row = h_kv * d_h elements of elem_bytes.

@@ -12,7 +12,12 @@
 //
 // Kernels:  dots (norms + next-frame dot, one warp per token)  ->  spatial (one CTA per crop)  ->
 //           fuse (one CTA per frame: s_temp, three standardisations, sum)  ->  topk (one CTA per sequence,
-//           8-bit radix select on order-preserving keys, ordered compaction).
+//           bisection on order-preserving keys, ordered compaction).
+//
+// hippo_select_tokens_policy adds the selection rules the paper compares itself with, as rules only: a uniform budget
+// per frame (the attention-guided uniform pruning of earlier video speculative decoding, related-work section), the k
+// best by caller-supplied random keys and whole frames at a regular stride (exploration of pruning criteria,
+// Section 6).  Uniform: budgets by one thread per sequence, then one CTA per frame ranks its tokens by counting.
 #include <math.h>
 
 #include "common.cuh"
@@ -34,6 +39,8 @@ struct SelectParams {
     int frame_off[kSelMaxBatch + 1];  // frame offset of each sequence
     int k[kSelMaxBatch];
     int k_off[kSelMaxBatch + 1];
+    int *frame_budget;               // per-frame policy: [frames] tokens kept / [frames] first output position
+    int *frame_out;
 };
 
 __device__ __forceinline__ double ld_as_double(const float *p, size_t i) { return (double)p[i]; }
@@ -445,14 +452,90 @@ __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p,
     }
 }
 
-struct SelectWs { size_t norm2_off, tdot_off, spa_off, total; };
-static SelectWs select_ws(long long total_tokens) {
+// ---- uniform budget per frame ------------------------------------------------------------------------------------
+// Budgets of one sequence, by one thread: floor(k / F) per frame, the first k mod F frames one more; a frame with fewer
+// tokens than its budget keeps them all and the shortfall goes, one token at a time in frame order, to the frames that
+// still have room.  Also the first output position of every frame.
+__global__ void select_budget_kernel(const SelectParams p) {
+    const int b = blockIdx.x;
+    if (threadIdx.x != 0) return;
+    const int n = p.seq_off[b + 1] - p.seq_off[b], k = p.k[b];
+    const int F = (n + p.tpf - 1) / p.tpf;
+    int *budget = p.frame_budget + p.frame_off[b], *first = p.frame_out + p.frame_off[b];
+    int given = 0;
+    for (int f = 0; f < F; ++f) {
+        const int want = k / F + (f < k % F ? 1 : 0), have = min(p.tpf, n - f * p.tpf);
+        budget[f] = min(want, have);
+        given += budget[f];
+    }
+    while (given < k)
+        for (int f = 0; f < F && given < k; ++f)
+            if (budget[f] < min(p.tpf, n - f * p.tpf)) { ++budget[f]; ++given; }
+    int acc = 0;
+    for (int f = 0; f < F; ++f) { first[f] = acc; acc += budget[f]; }
+}
+
+// One CTA per frame, thread c owns grid cell c: its rank among the frame's tokens by (score as fp32 descending, index
+// ascending) is a count over the frame's keys in shared memory; the kept ones are written in index order.
+__global__ void __launch_bounds__(1024) select_frame_topk_kernel(const SelectParams p) {
+    __shared__ uint32_t keys[1024];
+    __shared__ int warp_cnt[32];
+    const int gframe = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = find_seq(p.frame_off, p.batch, gframe);
+    const int f = gframe - p.frame_off[b];
+    const int n_v = p.seq_off[b + 1] - p.seq_off[b];
+    const int nf = min(p.tpf, n_v - f * p.tpf);
+    const int kf = p.frame_budget[gframe];
+    const bool valid = tid < nf;
+    const uint32_t key = valid ? order_key(p.fused[p.seq_off[b] + f * p.tpf + tid]) : 0u;
+    keys[tid] = key;
+    __syncthreads();
+    int rank = 0;
+    for (int c = 0; c < nf; ++c) {
+        const uint32_t other = keys[c];
+        rank += (other > key || (other == key && c < tid)) ? 1 : 0;
+    }
+    const bool sel = valid && rank < kf;
+    const unsigned bal = __ballot_sync(0xffffffffu, sel);
+    if (lane == 0) warp_cnt[warp] = __popc(bal);
+    __syncthreads();
+    int before = __popc(bal & ((1u << lane) - 1));
+    for (int w = 0; w < warp; ++w) before += warp_cnt[w];
+    if (sel) p.kept[p.k_off[b] + p.frame_out[gframe] + before] = f * p.tpf + tid;
+}
+
+// ---- whole frames at a regular stride --------------------------------------------------------------------------------
+// Output position i of sequence b: with m = ceil(k / T) frames kept out of the Fc complete ones, frame floor(q * Fc / m)
+// for q = i / T, cell i mod T (the last kept frame is cut short when k is not a multiple of T); when k reaches Fc * T, or
+// there is no complete frame, the first k tokens.
+__global__ void select_frames_kernel(const SelectParams p) {
+    const int b = blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int k = p.k[b];
+    if (i >= k) return;
+    const int n = p.seq_off[b + 1] - p.seq_off[b], T = p.tpf, Fc = n / T;
+    int idx = i;
+    if (Fc > 0 && (long long)k < (long long)Fc * T) {
+        const int m = (k + T - 1) / T;
+        idx = (int)((long long)(i / T) * Fc / m) * T + i % T;
+    }
+    p.kept[p.k_off[b] + i] = idx;
+}
+
+__global__ void select_copy_keys_kernel(const float *keys, float *fused, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) fused[i] = keys[i];
+}
+
+struct SelectWs { size_t norm2_off, tdot_off, spa_off, budget_off, total; };
+static SelectWs select_ws(long long total_tokens, long long total_frames) {
     SelectWs w;
     const size_t a = align_up((size_t)total_tokens * sizeof(double), 256);
     w.norm2_off = kWsHeaderBytes;
     w.tdot_off = w.norm2_off + a;
     w.spa_off = w.tdot_off + a;
-    w.total = w.spa_off + a;
+    w.budget_off = w.spa_off + a;       // per-frame policy: budget and first output position of every frame
+    w.total = w.budget_off + align_up((size_t)total_frames * 2 * sizeof(int), 256);
     return w;
 }
 
@@ -462,11 +545,12 @@ extern "C" {
 
 size_t hippo_select_workspace_bytes(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w,
                                     int32_t crop_h, int32_t crop_w) {
-    (void)grid_h; (void)grid_w; (void)crop_h; (void)crop_w;
-    if (batch <= 0 || !n_visual) return 0;
-    long long t = 0;
-    for (int b = 0; b < batch; ++b) { if (n_visual[b] <= 0) return 0; t += n_visual[b]; }
-    return hippo::select_ws(t).total;
+    (void)crop_h; (void)crop_w;
+    if (batch <= 0 || !n_visual || grid_h <= 0 || grid_w <= 0) return 0;
+    long long t = 0, f = 0;
+    const long long tpf = (long long)grid_h * grid_w;
+    for (int b = 0; b < batch; ++b) { if (n_visual[b] <= 0) return 0; t += n_visual[b]; f += (n_visual[b] + tpf - 1) / tpf; }
+    return hippo::select_ws(t, f).total;
 }
 
 int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w, int32_t crop_h,
@@ -474,9 +558,22 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
                             const float *attn_mass, const int32_t *k, const int32_t *kept_offsets,
                             uint32_t score_mask, int32_t *kept_idx, float *fused_score, void *workspace,
                             size_t workspace_bytes, void *stream) {
+    return hippo_select_tokens_policy(batch, n_visual, grid_h, grid_w, crop_h, crop_w, embed_dim, dtype, embeds, attn_mass, k,
+                                      kept_offsets, score_mask, HIPPO_SELECT_HOLISTIC, nullptr, kept_idx, fused_score,
+                                      workspace, workspace_bytes, stream);
+}
+
+int32_t hippo_select_tokens_policy(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w, int32_t crop_h,
+                                   int32_t crop_w, int32_t embed_dim, int32_t dtype, const void *embeds,
+                                   const float *attn_mass, const int32_t *k, const int32_t *kept_offsets,
+                                   uint32_t score_mask, int32_t policy, const float *random_keys, int32_t *kept_idx,
+                                   float *fused_score, void *workspace, size_t workspace_bytes, void *stream) {
     using namespace hippo;
     const char *who = "hippo_select_tokens";
     if (batch <= 0 || !n_visual || !k) return fail(HIPPO_ERR_INVALID_ARG, "%s: bad batch / null host arrays", who);
+    if (policy < HIPPO_SELECT_HOLISTIC || policy > HIPPO_SELECT_FRAMES) return fail(HIPPO_ERR_INVALID_ARG, "%s: unknown policy %d", who, policy);
+    const bool scored = policy == HIPPO_SELECT_HOLISTIC || policy == HIPPO_SELECT_UNIFORM_PER_FRAME;
+    if (policy == HIPPO_SELECT_RANDOM && !random_keys) return fail(HIPPO_ERR_INVALID_ARG, "%s: the random policy needs random_keys", who);
     if (batch > kSelMaxBatch) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: batch > %d", who, kSelMaxBatch);
     if (grid_h <= 0 || grid_w <= 0 || crop_h <= 0 || crop_w <= 0 || embed_dim <= 0)
         return fail(HIPPO_ERR_INVALID_ARG, "%s: non-positive geometry", who);
@@ -484,10 +581,11 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
     if (crop_h * crop_w > kMaxCrop) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: crop larger than %d tokens", who, kMaxCrop);
     if ((long long)grid_h * grid_w > 1024) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: more than 1024 tokens per frame", who);
     if (embed_dim % 8) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: embed_dim must be a multiple of 8", who);
-    if (!embeds || !attn_mass || !fused_score || !workspace) return fail(HIPPO_ERR_INVALID_ARG, "%s: null pointer", who);
+    if (!workspace || (scored && (!embeds || !attn_mass)) || (policy != HIPPO_SELECT_FRAMES && !fused_score))
+        return fail(HIPPO_ERR_INVALID_ARG, "%s: null pointer", who);
     if ((score_mask & ~HIPPO_SCORE_ALL) != 0) return fail(HIPPO_ERR_INVALID_ARG, "%s: unknown score_mask bits", who);
     if ((uintptr_t)workspace & 255) return fail(HIPPO_ERR_INVALID_ARG, "%s: workspace must be 256-byte aligned", who);
-    if ((uintptr_t)embeds & 15) return fail(HIPPO_ERR_INVALID_ARG, "%s: embeds must be 16-byte aligned", who);
+    if (scored && ((uintptr_t)embeds & 15)) return fail(HIPPO_ERR_INVALID_ARG, "%s: embeds must be 16-byte aligned", who);
 
     SelectParams p;
     p.tpf = grid_h * grid_w;
@@ -503,17 +601,35 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
     }
     p.seq_off[batch] = (int)tok; p.frame_off[batch] = (int)frames; p.k_off[batch] = (int)ksum;
     if (ksum > 0 && !kept_idx) return fail(HIPPO_ERR_INVALID_ARG, "%s: null kept_idx", who);
-    SelectWs w = select_ws(tok);
+    SelectWs w = select_ws(tok, frames);
     if (workspace_bytes < w.total) return fail(HIPPO_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu bytes", who, workspace_bytes, w.total);
     p.embeds = embeds; p.attn_mass = attn_mass; p.fused = fused_score; p.kept = kept_idx;
     p.norm2 = (double *)((char *)workspace + w.norm2_off);
     p.tdot = (double *)((char *)workspace + w.tdot_off);
     p.s_spa = (double *)((char *)workspace + w.spa_off);
+    p.frame_budget = (int *)((char *)workspace + w.budget_off);
+    p.frame_out = p.frame_budget + frames;
     p.batch = batch; p.grid_h = grid_h; p.grid_w = grid_w; p.crop_h = crop_h; p.crop_w = crop_w; p.d = embed_dim;
     p.crops_y = ceil_div(grid_h, crop_h); p.crops_x = ceil_div(grid_w, crop_w);
     p.mask = score_mask;
     cudaStream_t s = (cudaStream_t)stream;
-    const bool need_emb = (score_mask & (HIPPO_SCORE_TEMP | HIPPO_SCORE_SPA)) != 0;
+    if (policy == HIPPO_SELECT_FRAMES) {
+        // an index rule: no scores are formed, fused_score is not written
+        int kmax = 0;
+        for (int b = 0; b < batch; ++b) kmax = k[b] > kmax ? k[b] : kmax;
+        if (kmax > 0) {
+            select_frames_kernel<<<dim3((unsigned)ceil_div(kmax, 256), (unsigned)batch), 256, 0, s>>>(p);
+            count_launches(1);
+        }
+        HIPPO_CUDA_TRY(cudaGetLastError());
+        return HIPPO_OK;
+    }
+    if (policy == HIPPO_SELECT_RANDOM) {
+        // the caller's keys take the place of the fused score (and are returned as such)
+        select_copy_keys_kernel<<<(unsigned)((tok + 255) / 256), 256, 0, s>>>(random_keys, fused_score, (int)tok);
+        count_launches(1);
+    }
+    const bool need_emb = scored && (score_mask & (HIPPO_SCORE_TEMP | HIPPO_SCORE_SPA)) != 0;
     if (need_emb) {
         const int warps = 8;
         dim3 g1((unsigned)((tok + warps - 1) / warps));
@@ -521,7 +637,7 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
         else select_dots_kernel<__nv_bfloat16><<<g1, warps * 32, 0, s>>>(p);
         count_launches(1);
     }
-    if (score_mask & HIPPO_SCORE_SPA) {
+    if (scored && (score_mask & HIPPO_SCORE_SPA)) {
         dim3 g2((unsigned)(frames * p.crops_y * p.crops_x));
         static PerDeviceOnce spa_attr;
         int dev;
@@ -542,9 +658,15 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
         count_launches(1);
     }
     const int fuse_threads = ((p.tpf + 31) / 32) * 32;
-    select_fuse_kernel<<<(unsigned)frames, fuse_threads, 0, s>>>(p);
-    count_launches(1);
-    if (ksum > 0) {
+    if (scored) {
+        select_fuse_kernel<<<(unsigned)frames, fuse_threads, 0, s>>>(p);
+        count_launches(1);
+    }
+    if (ksum > 0 && policy == HIPPO_SELECT_UNIFORM_PER_FRAME) {
+        select_budget_kernel<<<batch, 32, 0, s>>>(p);
+        select_frame_topk_kernel<<<(unsigned)frames, fuse_threads, 0, s>>>(p);
+        count_launches(2);
+    } else if (ksum > 0) {
         // shared-memory staging for the keys beyond 32 per thread, up to 48K of them
         int longest = 0;
         for (int b = 0; b < batch; ++b) longest = n_visual[b] > longest ? n_visual[b] : longest;

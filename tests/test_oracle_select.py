@@ -205,3 +205,71 @@ def test_config0_keep_count_and_boundary_share():
     idx, fused, kth = oracle.select_tokens(inp["embeds"], inp["attn_mass"], inp["k"], 8, 8)
     assert len(idx) == 26 and np.all(np.diff(idx) > 0)
     assert np.all(fused[idx] >= kth) and np.sum(fused > kth) <= 26
+
+
+# ---- the other selection rules (uniform per-frame budget, random keys, whole frames) --------------------------------
+
+def test_policy_per_frame_budgets_and_in_frame_order():
+    """Uniform pruning across frames: budgets worked by hand, and inside each frame numpy's stable arg-sort."""
+    rng = np.random.default_rng(31)
+    T = 12
+    # 5 complete frames, k = 17: 17 // 5 = 3 each, the first 17 % 5 = 2 frames one more
+    s = rng.standard_normal(5 * T)
+    kept, budget = oracle.select_policy(oracle.POLICY_UNIFORM_PER_FRAME, s, 17, T)
+    assert budget.tolist() == [4, 4, 3, 3, 3]
+    want = np.concatenate([f * T + np.sort(np.argsort(-s[f * T:(f + 1) * T], kind="stable")[:budget[f]]) for f in range(5)])
+    assert kept.tolist() == want.tolist()
+    assert np.all(np.diff(kept) > 0)
+    # k divisible by the frame count: the same share everywhere; k = 0; k = n keeps everything
+    assert oracle.select_policy(1, s, 20, T)[1].tolist() == [4] * 5
+    assert oracle.select_policy(1, s, 0, T)[0].size == 0
+    assert oracle.select_policy(1, s, 5 * T, T)[0].tolist() == list(range(5 * T))
+    # a partial last frame of 2 tokens with k = 16 over 4 frames: 4 each, the last can give 2, the shortfall of 2 goes
+    # to frames 0 and 1 in order
+    s2 = rng.standard_normal(3 * T + 2)
+    kept, budget = oracle.select_policy(1, s2, 16, T)
+    assert budget.tolist() == [5, 5, 4, 2]
+    assert kept[-2:].tolist() == [3 * T, 3 * T + 1]
+    # shortfall larger than one round: frames 0..2 of 12, a partial frame of 1 token, k = 34 -> 9, 9, 8, 8 wanted;
+    # the last gives 1, 7 missing: +1 each to frames 0, 1, 2 twice (12 = full for none yet), then +1 to frame 0
+    s3 = rng.standard_normal(3 * T + 1)
+    assert oracle.select_policy(1, s3, 34, T)[1].tolist() == [12, 11, 10, 1]
+    # one frame: the per-frame rule is the global rule
+    one = rng.standard_normal(T)
+    assert oracle.select_policy(1, one, 5, T)[0].tolist() == oracle.select_policy(0, one, 5, T)[0].tolist()
+    # ties inside a frame: the lowest indices win
+    flat = np.zeros(2 * T)
+    assert oracle.select_policy(1, flat, 6, T)[0].tolist() == [0, 1, 2, T, T + 1, T + 2]
+
+
+def test_policy_random_is_the_top_k_of_the_callers_keys():
+    rng = np.random.default_rng(32)
+    keys = rng.random(500).astype(np.float32)
+    keys[[7, 300]] = keys[11]                                           # equal keys: the lower index first
+    for k in (0, 1, 50, 499, 500):
+        kept, _ = oracle.select_policy(oracle.POLICY_RANDOM, keys, k, 25)
+        want = np.sort(np.lexsort((np.arange(500), -keys.astype(np.float64)))[:k])
+        assert kept.tolist() == want.tolist()
+
+
+def test_policy_whole_frames_at_a_regular_stride():
+    T = 4
+    none = np.zeros(8 * T)
+    # 8 frames, keep 2 whole frames: frames 0 and 4; keep 4: frames 0, 2, 4, 6
+    assert oracle.select_policy(oracle.POLICY_FRAME, none, 2 * T, T)[0].tolist() == [0, 1, 2, 3, 16, 17, 18, 19]
+    kept = oracle.select_policy(3, none, 4 * T, T)[0]
+    assert sorted(set((kept // T).tolist())) == [0, 2, 4, 6] and kept.size == 16
+    # 3 frames out of 8: floor(i * 8 / 3) = 0, 2, 5
+    assert sorted(set((oracle.select_policy(3, none, 3 * T, T)[0] // T).tolist())) == [0, 2, 5]
+    # k not a multiple of the frame size: ceil(10 / 4) = 3 frames 0, 2, 5, the last one cut to its first 2 cells
+    assert oracle.select_policy(3, none, 10, T)[0].tolist() == [0, 1, 2, 3, 8, 9, 10, 11, 20, 21]
+    # every complete frame and more: a prefix of the sequence (partial last frame of 3 cells)
+    part = np.zeros(2 * T + 3)
+    assert oracle.select_policy(3, part, 2 * T + 1, T)[0].tolist() == list(range(9))
+    assert oracle.select_policy(3, part, 5, T)[0].tolist() == [0, 1, 2, 3, 4]      # ceil(5/4) = 2 frames of 2: 0 and 1, second cut
+    # no complete frame at all
+    assert oracle.select_policy(3, np.zeros(3), 2, T)[0].tolist() == [0, 1]
+    # ascending, exactly k, for a sweep
+    for k in range(0, 8 * T + 1):
+        kept = oracle.select_policy(3, none, k, T)[0]
+        assert kept.size == k and np.all(np.diff(kept) > 0)

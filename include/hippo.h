@@ -14,12 +14,14 @@
  *     host before anything is enqueued; on an error nothing has been launched.
  *   - Pointers are DEVICE pointers unless the comment says "host".  The caller owns every buffer, including
  *     workspaces (size them with the *_workspace_bytes helpers; 256-byte aligned).  The library allocates
- *     no device memory and keeps no state between calls besides a per-thread error string and cached
- *     kernel attributes.
+ *     no device memory.  Between calls it keeps a per-thread error string, cached kernel attributes, and - for
+ *     hippo_accept_noalloc alone - a fixed scratch array in its image (HIPPO_ACCEPT_NOALLOC_SCRATCH_BYTES on every
+ *     GPU that loads the library) with that array's cached address.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*) and the call returns without synchronising.
  *     Calls on different streams may overlap if they use different workspaces and outputs.
- *   - Device-side waits are bounded.  If one gives up, the kernel records it in the first word of the
- *     workspace and exits; hippo_workspace_status() reports it after the stream has drained.
+ *   - Device-side waits are bounded (2 s).  If one gives up, the kernel records it in the first word of the
+ *     workspace, waits for its own copies and tensor-core work in flight, frees its tensor memory and exits;
+ *     hippo_workspace_status() reports it after the stream has drained.  Results of that call are undefined.
  *   - dtype: HIPPO_DTYPE_FP32 or HIPPO_DTYPE_BF16 storage; accumulation is fp32 (attention) or fp64
  *     (selection scores, acceptance).
  */
@@ -33,7 +35,7 @@
 extern "C" {
 #endif
 
-#define HIPPO_VERSION 100
+#define HIPPO_VERSION 101
 #define HIPPO_PAGE_SIZE 64          /* tokens per KV page */
 #define HIPPO_MAX_PACKED_ROWS 128   /* q_len * (n_q_heads / n_kv_heads) must not exceed this */
 
@@ -50,6 +52,14 @@ typedef enum hippo_status {
 typedef enum hippo_dtype { HIPPO_DTYPE_FP32 = 0, HIPPO_DTYPE_BF16 = 1 } hippo_dtype_t;
 
 typedef enum hippo_accept_mode { HIPPO_ACCEPT_SAMPLE = 0, HIPPO_ACCEPT_GREEDY = 1 } hippo_accept_mode_t;
+
+/* selection rules of hippo_select_tokens_policy */
+typedef enum hippo_select_policy {
+    HIPPO_SELECT_HOLISTIC = 0,            /* Section 5.1: the k best of the fused score over the whole sequence */
+    HIPPO_SELECT_UNIFORM_PER_FRAME = 1,   /* the same budget for every frame, the best of the fused score inside each */
+    HIPPO_SELECT_RANDOM = 2,              /* the k best by a caller-supplied random key per token */
+    HIPPO_SELECT_FRAMES = 3               /* whole frames at a regular stride */
+} hippo_select_policy_t;
 
 /* score_mask bits for hippo_select_tokens (Eq. 7 sums the enabled terms) */
 #define HIPPO_SCORE_ATTN 1u
@@ -89,9 +99,20 @@ uint64_t hippo_launch_count(void);
 /* Synchronises `stream`, then reads the status word that kernels keep in the first bytes of `workspace`:
  * HIPPO_OK, or HIPPO_ERR_TIMEOUT if a bounded device-side wait gave up since hippo_workspace_reset(). */
 int32_t hippo_workspace_status(const void *workspace, void *stream);
-/* Zeroes the header of a workspace (status word and arrival counters); enqueued on `stream`.  Must be called
- * once on a fresh workspace before its first use by the attention calls, and after a reported time-out. */
+/* Zeroes the header of a workspace (status word, wait limit and arrival counters); enqueued on `stream`.  Must be
+ * called once on a fresh workspace before its first use by the attention calls, and after a reported time-out. */
 int32_t hippo_workspace_reset(void *workspace, size_t workspace_bytes, void *stream);
+/* Debugging aid: replaces the 2 s limit of the bounded device-side waits of the tensor-core attention and
+ * attention-mass kernels that use this workspace by `limit_ns` nanoseconds (0 restores the default).  The waits that
+ * guard a kernel's exit (its own copies and tensor-core work in flight) keep the 2 s limit.  Synchronises `stream`.
+ * With a limit of a few microseconds a healthy kernel gives up on its first wait: this is how the time-out path
+ * (status word, clean exit, reset) can be exercised without anything being stuck. */
+int32_t hippo_workspace_set_wait_limit(void *workspace, int64_t limit_ns, void *stream);
+
+/* Measurement aid (no counterpart in the paper): one pass of 16-byte loads over `bytes` bytes at `buffer`, summed into
+ * `sink` (256 bytes of device memory, 256-byte aligned; contents are a checksum of no interest).  Timed by the caller,
+ * it gives the bandwidth a read-only kernel reaches on this device, the natural ceiling of the attention kernels. */
+int32_t hippo_read_probe(const void *buffer, size_t bytes, void *sink, void *stream);
 
 /* ---- global semantic relevance: Section 5.1, Eq. 2 ------------------------------------------------------------ */
 /*
@@ -143,36 +164,73 @@ int32_t hippo_select_tokens(int32_t batch, const int32_t *n_visual, int32_t grid
                             uint32_t score_mask, int32_t *kept_idx, float *fused_score, void *workspace,
                             size_t workspace_bytes, void *stream);
 
-/* ---- gather: pruning the draft KV cache (Limitations (i); experimental set-up: "remove the corresponding
- *      video features") --------------------------------------------------------------------------------------- */
+/*
+ * hippo_select_tokens under another selection rule.  The paper contrasts its holistic top-k with uniform pruning across
+ * frames guided by the target's attention (related work on video speculative decoding) and, in its exploration of
+ * pruning criteria (Section 6), with randomly sampled tokens and with whole frames dropped at regular temporal intervals;
+ * it names these rules without spelling them out, so the definitions below are this library's reading.  Rules only:
+ * the comparison systems themselves are not part of the library.
+ *   HIPPO_SELECT_HOLISTIC           exactly hippo_select_tokens.
+ *   HIPPO_SELECT_UNIFORM_PER_FRAME  the fused score as above (score_mask = HIPPO_SCORE_ATTN gives attention-guided uniform
+ *                                   pruning); frame f of F keeps floor(k / F) tokens, the first k mod F frames one more;
+ *                                   a frame with fewer tokens than its budget (a partial last frame) keeps them all and
+ *                                   the shortfall goes, one token at a time in frame order, to frames that still have room;
+ *                                   inside a frame the best by (fused as fp32 descending, index ascending).
+ *   HIPPO_SELECT_RANDOM             random_keys (fp32 [sum n_visual], drawn by the caller) take the place of the fused
+ *                                   score: the k best keys over the sequence, lower index first among equal keys.
+ *                                   fused_score receives the keys.  embeds and attn_mass are not read and may be NULL.
+ *   HIPPO_SELECT_FRAMES             with T = grid_h * grid_w, Fc = n_visual / T complete frames and m = ceil(k / T):
+ *                                   frames floor(i * Fc / m), i = 0 .. m-1, whole, the last of them cut to its first cells
+ *                                   when k is not a multiple of T; if k >= Fc * T (or Fc = 0) the first k tokens.
+ *                                   Nothing is scored: embeds, attn_mass and fused_score are not touched and may be NULL.
+ * All other arguments, the output order (ascending per sequence) and the workspace are those of hippo_select_tokens.
+ */
+int32_t hippo_select_tokens_policy(int32_t batch, const int32_t *n_visual, int32_t grid_h, int32_t grid_w, int32_t crop_h,
+                                   int32_t crop_w, int32_t embed_dim, int32_t dtype, const void *embeds,
+                                   const float *attn_mass, const int32_t *k, const int32_t *kept_offsets,
+                                   uint32_t score_mask, int32_t policy, const float *random_keys, int32_t *kept_idx,
+                                   float *fused_score, void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- gather: pruning the draft KV cache (Limitations (i); the experimental set-up drops the pruned tokens'
+ *      features from the draft model's input) ------------------------------------------------------------------- */
 /*
  * For every layer l < n_layers, sequence b and i in [keep_offsets[b], keep_offsets[b+1]):
  *     dst token (i - keep_offsets[b]) of sequence b  :=  src token keep_idx[i] of sequence b      (K and V, all heads)
  * `src` / `dst` describe layer 0; layer l's pools start src_layer_stride_bytes * l (dst_layer_stride_bytes * l)
  * bytes further on.  Page tables are shared by all layers.  keep_idx holds positions in the source sequence
  * (the kept visual tokens and every always-kept position such as text), ascending per sequence to preserve
- * order; the kernel does not require ascending order.  Indices are not range-checked on the device: the
- * caller guarantees 0 <= keep_idx < source length.  src and dst must not overlap and must agree in dtype,
+ * order; the kernel does not require ascending order.  src and dst must not overlap and must agree in dtype,
  * n_kv_heads and head_dim (head_dim * element size a multiple of 16 bytes).
+ * Indices are read on the device and checked there before any address is formed from them: a source position
+ * outside [0, src max_pages_per_seq * 64), a destination position beyond dst max_pages_per_seq * 64 (a sequence
+ * keeping more than its destination holds), or a page id outside [0, n_pages) of its pool.  Such an entry is
+ * skipped (nothing is read or written for it) and *bad_index is set to 1.  A source position inside the page
+ * capacity but past the sequence's length copies whatever the slot holds.
  *   keep_idx      int32 [total_keep]          keep_offsets  int32 [batch + 1] (device), keep_offsets[0] = 0
- *   total_keep    host copy of keep_offsets[batch]
+ *   total_keep    host copy of keep_offsets[batch]; must not exceed batch * dst max_pages_per_seq * 64
+ *   bad_index     optional device int32, zeroed by the caller; NULL: bad entries are skipped silently
  */
 int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src, size_t src_layer_stride_bytes,
                         const hippo_kv_cache_t *dst, size_t dst_layer_stride_bytes, int32_t batch,
-                        const int32_t *keep_idx, const int32_t *keep_offsets, int32_t total_keep, void *stream);
+                        const int32_t *keep_idx, const int32_t *keep_offsets, int32_t total_keep,
+                        int32_t *bad_index, void *stream);
 
 /* ---- attention: Section 3.2 (drafting phase / verification phase) ------------------------------------------ */
 /*
  * out[b][t][h] = softmax_j( scale * q[b][t][h] . K[b][j][h / G] ) V[b][j][h / G],   G = n_q_heads / n_kv_heads,
  * over the keys j <= kv_len[b] - q_len + t: the q_len query tokens are the LAST q_len positions of the
  * kv_len[b]-token context (their own K/V are already in the cache), every earlier key is visible.
- * hippo_verify_attention is tuned for q_len = gamma + 1 rows against the full-length video cache (one persistent
- * CTA per SM streaming K/V tiles); hippo_draft_attention for q_len = 1 against the short pruned cache
- * (many small splits).  Both compute the same function for any q_len >= 1.
+ * The verification call is q_len = gamma + 1 rows against the full-length video cache, the draft call q_len = 1
+ * against the short pruned cache.  Both names compute the same function for any q_len >= 1 and pick the kernel from
+ * the shape: up to 8 packed rows over at most 1,024 keys run as one cluster of CTAs with a page each (latency-bound);
+ * anything larger streams K/V tiles through one persistent CTA per SM.
  *   q        [batch][q_len][n_q_heads][head_dim] dtype        out  same shape and dtype as q
  *   kv_len   int32 [batch] (device), q_len <= kv_len[b] <= max_kv_len;  a sequence with kv_len[b] < q_len is skipped.
  *            NULL means the lengths are known on the host and all equal max_kv_len: the kernels then start their
  *            loads without the round trip for the length
+ *   kv_len_host  optional HOST copy of kv_len (NULL: none).  Used only to plan the launch: with the real lengths of a
+ *            ragged batch the work split is chosen from the total number of pages instead of batch * the longest;
+ *            the kernels still read kv_len on the device, results do not depend on it
  *   max_kv_len  host upper bound used to size the launch; <= max_pages_per_seq * 64
  *   softmax_scale  0 selects 1/sqrt(head_dim)
  *   num_splits  0 = automatic
@@ -184,13 +242,41 @@ int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src, size_t sr
 size_t hippo_attention_workspace_bytes(int32_t batch, int32_t q_len, int32_t n_q_heads, int32_t n_kv_heads,
                                        int32_t head_dim);
 int32_t hippo_verify_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, const void *q,
-                               const hippo_kv_cache_t *kv, const int32_t *kv_len, int32_t max_kv_len,
-                               float softmax_scale, int32_t num_splits, void *out, float *lse, void *workspace,
-                               size_t workspace_bytes, void *stream);
+                               const hippo_kv_cache_t *kv, const int32_t *kv_len, const int32_t *kv_len_host,
+                               int32_t max_kv_len, float softmax_scale, int32_t num_splits, void *out, float *lse,
+                               void *workspace, size_t workspace_bytes, void *stream);
 int32_t hippo_draft_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, const void *q,
-                              const hippo_kv_cache_t *kv, const int32_t *kv_len, int32_t max_kv_len,
-                              float softmax_scale, int32_t num_splits, void *out, float *lse, void *workspace,
-                              size_t workspace_bytes, void *stream);
+                              const hippo_kv_cache_t *kv, const int32_t *kv_len, const int32_t *kv_len_host,
+                              int32_t max_kv_len, float softmax_scale, int32_t num_splits, void *out, float *lse,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The verification attention of SEVERAL layers in one launch (Section 3.2, verification phase; the target model's
+ * verification pass runs this op once per layer over that layer's cache).  Same function as n_layers calls of
+ * hippo_verify_attention:  out_layers[l] = attention(q_layers[l], kv_layers[l])  for l in [0, n_layers).
+ * The persistent CTAs walk the layers: barriers, tensor memory and the work split are set up once, the loads of
+ * layer l + 1 start while the softmax of layer l finishes, and the partial results of a layer are merged by a spare
+ * warp of every CTA while the next layer streams, so no kernel boundary and no second kernel separate two layers.
+ * All layers share batch, q_len, heads, head_dim, dtype, kv_len and the page table (kv_layers[l].page_table must be the
+ * same pointer for every l, as must max_pages_per_seq; pools and n_pages may differ).
+ *   q_layers, out_layers   HOST arrays [n_layers] of DEVICE pointers, each [batch][q_len][n_q_heads][head_dim]
+ *   kv_layers              HOST array [n_layers] of descriptors
+ *   lse_layers             NULL, or HOST array [n_layers] of DEVICE pointers (entries may be NULL)
+ *   kv_len, kv_len_host, max_kv_len, softmax_scale   as for hippo_verify_attention
+ * The host arrays are read before the call returns.  The call enqueues one memset of its counters and one kernel
+ * per 64 layers.  The workspace is larger than a single-layer one (three sets of partial-result slots and per-layer
+ * counters): size it with hippo_verify_attention_layers_workspace_bytes.  bf16 with head_dim 64 or 128 and at most
+ * 256 (sequence, kv head) units use the multi-layer kernel; every other shape is run layer by layer on the
+ * single-layer paths, with the same results.  Because the CTAs of the launch wait for one another's partial results,
+ * the grid never exceeds the number of SMs; the waits are bounded like every other.
+ */
+size_t hippo_verify_attention_layers_workspace_bytes(int32_t n_layers, int32_t batch, int32_t q_len, int32_t n_q_heads,
+                                                     int32_t n_kv_heads, int32_t head_dim);
+int32_t hippo_verify_attention_layers(int32_t n_layers, int32_t batch, int32_t q_len, int32_t n_q_heads,
+                                      const void *const *q_layers, const hippo_kv_cache_t *kv_layers,
+                                      const int32_t *kv_len, const int32_t *kv_len_host, int32_t max_kv_len,
+                                      float softmax_scale, void *const *out_layers, float *const *lse_layers,
+                                      void *workspace, size_t workspace_bytes, void *stream);
 
 /* ---- acceptance: Section 3.2, Eq. 1 -------------------------------------------------------------------------- */
 /*
@@ -205,7 +291,8 @@ int32_t hippo_draft_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, c
  * Setups"): x_{j+1} is kept iff it equals the arg-max of target row j (lowest token id on ties); the emitted token
  * is the arg-max of target row n.  draft_logits, u_accept and u_resample are not read and may be NULL.
  *   target_logits fp32 [batch][gamma+1][vocab]     draft_logits fp32 [batch][gamma][vocab]
- *   draft_tokens  int32 [batch][gamma] in [0, vocab) u_accept fp32 [batch][gamma]    u_resample fp32 [batch]
+ *   draft_tokens  int32 [batch][gamma]; a token outside [0, vocab) is never looked up and counts as rejected
+ *   u_accept fp32 [batch][gamma]                    u_resample fp32 [batch]
  *   n_accepted    out int32 [batch]                 out_tokens out int32 [batch][gamma+1]: accepted draft tokens,
  *                                                   then the drawn token, then -1
  */
@@ -217,7 +304,7 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
 
 /*
  * hippo_accept for callers that cannot hand over a workspace.  (No counterpart in the paper: this is a packaging
- * variant of hippo_accept, same inputs, same outputs, same arithmetic.)
+ * variant of hippo_accept, same inputs, same outputs, same arithmetic, both modes.)
  *
  * Who needs it: code that reaches the acceptance step without any means of allocating device memory - a decode
  * loop whose memory was given in full to an engine's pool at start-up, a plug-in whose host forbids cudaMalloc

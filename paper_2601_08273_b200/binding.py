@@ -33,6 +33,7 @@ HIPPO_ERR_UNIMPLEMENTED = -6
 HIPPO_DTYPE_FP32 = 0
 HIPPO_DTYPE_BF16 = 1
 HIPPO_SCORE_ALL = 7
+HIPPO_SELECT_HOLISTIC, HIPPO_SELECT_UNIFORM_PER_FRAME, HIPPO_SELECT_RANDOM, HIPPO_SELECT_FRAMES = 0, 1, 2, 3
 HIPPO_ACCEPT_SAMPLE = 0
 HIPPO_ACCEPT_GREEDY = 1
 PAGE_SIZE = 64
@@ -58,18 +59,30 @@ lib.hippo_workspace_status.restype = _i32
 lib.hippo_workspace_status.argtypes = [_vp, _vp]
 lib.hippo_workspace_reset.restype = _i32
 lib.hippo_workspace_reset.argtypes = [_vp, _sz, _vp]
+lib.hippo_read_probe.restype = _i32
+lib.hippo_read_probe.argtypes = [_vp, _sz, _vp, _vp]
 lib.hippo_select_workspace_bytes.restype = _sz
 lib.hippo_select_workspace_bytes.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32]
 lib.hippo_select_tokens.restype = _i32
 lib.hippo_select_tokens.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _I32P, _I32P, _u32, _vp, _vp,
                                     _vp, _sz, _vp]
+lib.hippo_select_tokens_policy.restype = _i32
+lib.hippo_select_tokens_policy.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _I32P, _I32P, _u32, _i32, _vp,
+                                           _vp, _vp, _vp, _sz, _vp]
 lib.hippo_gather_kv.restype = _i32
-lib.hippo_gather_kv.argtypes = [_i32, _KVP, _sz, _KVP, _sz, _i32, _vp, _vp, _i32, _vp]
+lib.hippo_gather_kv.argtypes = [_i32, _KVP, _sz, _KVP, _sz, _i32, _vp, _vp, _i32, _vp, _vp]
 lib.hippo_attention_workspace_bytes.restype = _sz
 lib.hippo_attention_workspace_bytes.argtypes = [_i32] * 5
 for _name in ("hippo_verify_attention", "hippo_draft_attention"):
     getattr(lib, _name).restype = _i32
-    getattr(lib, _name).argtypes = [_i32, _i32, _i32, _vp, _KVP, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _sz, _vp]
+    getattr(lib, _name).argtypes = [_i32, _i32, _i32, _vp, _KVP, _vp, _I32P, _i32, _f32, _i32, _vp, _vp, _vp, _sz, _vp]
+lib.hippo_verify_attention_layers_workspace_bytes.restype = _sz
+lib.hippo_verify_attention_layers_workspace_bytes.argtypes = [_i32] * 6
+lib.hippo_verify_attention_layers.restype = _i32
+lib.hippo_verify_attention_layers.argtypes = [_i32, _i32, _i32, _i32, ctypes.POINTER(_vp), _KVP, _vp, _I32P, _i32, _f32,
+                                              ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _sz, _vp]
+lib.hippo_workspace_set_wait_limit.restype = _i32
+lib.hippo_workspace_set_wait_limit.argtypes = [_vp, ctypes.c_int64, _vp]
 lib.hippo_attention_mass_workspace_bytes.restype = _sz
 lib.hippo_attention_mass_workspace_bytes.argtypes = [_i32, _I32P, _i32, _i32, _i32, _i32, _i32]
 lib.hippo_attention_mass.restype = _i32
@@ -200,42 +213,71 @@ def hippo_workspace_reset(workspace: torch.Tensor, stream=None) -> None:
     _check(lib.hippo_workspace_reset(_ptr(workspace), workspace.numel(), _stream(stream)))
 
 
+def hippo_workspace_set_wait_limit(workspace: torch.Tensor, limit_ns: int, stream=None) -> None:
+    _check(lib.hippo_workspace_set_wait_limit(_ptr(workspace), int(limit_ns), _stream(stream)))
+
+
+def hippo_read_probe(buffer: torch.Tensor, sink: torch.Tensor, stream=None) -> None:
+    """One read-only pass over `buffer` (measurement aid); `sink`: 256 bytes of device memory."""
+    assert sink.numel() * sink.element_size() >= 256
+    _check(lib.hippo_read_probe(_ptr(buffer), buffer.numel() * buffer.element_size(), _ptr(sink), _stream(stream)))
+
+
 # ---- selection --------------------------------------------------------------------------------------------------
 
 def hippo_select_workspace_bytes(n_visual: Sequence[int], grid_h: int, grid_w: int, crop_h: int = 5, crop_w: int = 5) -> int:
     return int(lib.hippo_select_workspace_bytes(len(n_visual), _host_i32(n_visual), grid_h, grid_w, crop_h, crop_w))
 
 
-def hippo_select_tokens(embeds: torch.Tensor, attn_mass: torch.Tensor, n_visual: Sequence[int], k: Sequence[int],
-                        grid_h: int, grid_w: int, crop_h: int = 5, crop_w: int = 5, score_mask: int = HIPPO_SCORE_ALL,
-                        kept_idx: Optional[torch.Tensor] = None, kept_offsets: Optional[Sequence[int]] = None,
-                        fused_score: Optional[torch.Tensor] = None,
-                        workspace: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
-    """embeds [sum n_visual][d]; attn_mass fp32 [sum n_visual].  Returns (kept_idx int32 [sum k], fused fp32)."""
-    assert embeds.is_contiguous() and attn_mass.is_contiguous() and attn_mass.dtype == torch.float32
+def hippo_select_tokens(embeds: Optional[torch.Tensor], attn_mass: Optional[torch.Tensor], n_visual: Sequence[int],
+                        k: Sequence[int], grid_h: int, grid_w: int, crop_h: int = 5, crop_w: int = 5,
+                        score_mask: int = HIPPO_SCORE_ALL, kept_idx: Optional[torch.Tensor] = None,
+                        kept_offsets: Optional[Sequence[int]] = None, fused_score: Optional[torch.Tensor] = None,
+                        workspace: Optional[torch.Tensor] = None, stream=None, policy: int = HIPPO_SELECT_HOLISTIC,
+                        random_keys: Optional[torch.Tensor] = None, embed_dim: Optional[int] = None,
+                        device=None) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+    """embeds [sum n_visual][d]; attn_mass fp32 [sum n_visual].  Returns (kept_idx int32 [sum k], fused fp32).
+    policy != HIPPO_SELECT_HOLISTIC goes through hippo_select_tokens_policy (random_keys: fp32 [sum n_visual]); the
+    policies that score nothing accept embeds = attn_mass = None (then pass `device`)."""
     total = int(sum(n_visual))
-    assert embeds.shape[0] == total and attn_mass.shape[0] == total
+    if embeds is not None:
+        assert embeds.is_contiguous() and embeds.shape[0] == total
+        device, embed_dim = embeds.device, embeds.shape[1]
+    if attn_mass is not None:
+        assert attn_mass.is_contiguous() and attn_mass.dtype == torch.float32 and attn_mass.shape[0] == total
+    if random_keys is not None:
+        assert random_keys.is_contiguous() and random_keys.dtype == torch.float32 and random_keys.shape[0] == total
+        device = random_keys.device
+    device = torch.device("cuda") if device is None else device
     if kept_idx is None:
-        kept_idx = torch.empty(max(int(sum(k)), 1), dtype=torch.int32, device=embeds.device)
-    if fused_score is None:
-        fused_score = torch.empty(total, dtype=torch.float32, device=embeds.device)
+        kept_idx = torch.empty(max(int(sum(k)), 1), dtype=torch.int32, device=device)
+    if fused_score is None and policy != HIPPO_SELECT_FRAMES:
+        fused_score = torch.empty(total, dtype=torch.float32, device=device)
     if workspace is None:
-        workspace = new_workspace(hippo_select_workspace_bytes(n_visual, grid_h, grid_w, crop_h, crop_w), embeds.device)
-    _check(lib.hippo_select_tokens(len(n_visual), _host_i32(n_visual), grid_h, grid_w, crop_h, crop_w, embeds.shape[1],
-                                   _dtype_code(embeds), _ptr(embeds), _ptr(attn_mass), _host_i32(k),
-                                   None if kept_offsets is None else _host_i32(kept_offsets), score_mask,
-                                   _ptr(kept_idx), _ptr(fused_score), _ptr(workspace), workspace.numel(), _stream(stream)))
+        workspace = new_workspace(hippo_select_workspace_bytes(n_visual, grid_h, grid_w, crop_h, crop_w), device)
+    common = (len(n_visual), _host_i32(n_visual), grid_h, grid_w, crop_h, crop_w, 8 if embed_dim is None else int(embed_dim),
+              HIPPO_DTYPE_BF16 if embeds is None else _dtype_code(embeds), _ptr(embeds), _ptr(attn_mass), _host_i32(k),
+              None if kept_offsets is None else _host_i32(kept_offsets), score_mask)
+    tail = (_ptr(kept_idx), _ptr(fused_score), _ptr(workspace), workspace.numel(), _stream(stream))
+    if policy == HIPPO_SELECT_HOLISTIC and random_keys is None:
+        _check(lib.hippo_select_tokens(*common, *tail))
+    else:
+        _check(lib.hippo_select_tokens_policy(*common, int(policy), _ptr(random_keys), *tail))
     return (kept_idx[:int(sum(k))] if kept_offsets is None else kept_idx), fused_score
 
 
 # ---- gather -------------------------------------------------------------------------------------------------------
 
 def hippo_gather_kv(n_layers: int, src: KVCache, src_layer_stride_bytes: int, dst: KVCache, dst_layer_stride_bytes: int,
-                    batch: int, keep_idx: torch.Tensor, keep_offsets: torch.Tensor, total_keep: int, stream=None) -> None:
+                    batch: int, keep_idx: torch.Tensor, keep_offsets: torch.Tensor, total_keep: int,
+                    bad_index: Optional[torch.Tensor] = None, stream=None) -> None:
+    """bad_index: optional int32 device word (zeroed by the caller) that the kernel sets when it skipped an
+    out-of-range entry."""
     assert keep_idx.dtype == torch.int32 and keep_offsets.dtype == torch.int32
+    assert bad_index is None or bad_index.dtype == torch.int32
     _check(lib.hippo_gather_kv(n_layers, ctypes.byref(src.struct), src_layer_stride_bytes, ctypes.byref(dst.struct),
                                dst_layer_stride_bytes, batch, _ptr(keep_idx), _ptr(keep_offsets), int(total_keep),
-                               _stream(stream)))
+                               _ptr(bad_index), _stream(stream)))
 
 
 # ---- attention ----------------------------------------------------------------------------------------------------
@@ -244,7 +286,7 @@ def hippo_attention_workspace_bytes(batch: int, q_len: int, n_q_heads: int, n_kv
     return int(lib.hippo_attention_workspace_bytes(batch, q_len, n_q_heads, n_kv_heads, head_dim))
 
 
-def _attention(fn, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse, workspace, stream):
+def _attention(fn, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse, workspace, stream, kv_len_host=None):
     assert q.is_contiguous() and q.dim() == 4 and (kv_len is None or kv_len.dtype == torch.int32)
     B, q_len, hq, d = q.shape
     assert d == kv.head_dim and _dtype_code(q) == kv.struct.dtype
@@ -252,23 +294,58 @@ def _attention(fn, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, ls
         out = torch.empty_like(q)
     if workspace is None:
         workspace = new_workspace(hippo_attention_workspace_bytes(B, q_len, hq, kv.n_kv_heads, d), q.device)
-    _check(fn(B, q_len, hq, _ptr(q), ctypes.byref(kv.struct), _ptr(kv_len), int(max_kv_len), float(softmax_scale),
+    _check(fn(B, q_len, hq, _ptr(q), ctypes.byref(kv.struct), _ptr(kv_len),
+              None if kv_len_host is None else _host_i32(kv_len_host), int(max_kv_len), float(softmax_scale),
               int(num_splits), _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel(), _stream(stream)))
     return out
 
 
 def hippo_verify_attention(q: torch.Tensor, kv: KVCache, kv_len: torch.Tensor, max_kv_len: int,
                            softmax_scale: float = 0.0, num_splits: int = 0, out: Optional[torch.Tensor] = None,
-                           lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+                           lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None,
+                           kv_len_host: Optional[Sequence[int]] = None):
     return _attention(lib.hippo_verify_attention, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse,
-                      workspace, stream)
+                      workspace, stream, kv_len_host)
 
 
 def hippo_draft_attention(q: torch.Tensor, kv: KVCache, kv_len: torch.Tensor, max_kv_len: int,
                           softmax_scale: float = 0.0, num_splits: int = 0, out: Optional[torch.Tensor] = None,
-                          lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+                          lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None,
+                          kv_len_host: Optional[Sequence[int]] = None):
     return _attention(lib.hippo_draft_attention, q, kv, kv_len, max_kv_len, softmax_scale, num_splits, out, lse,
-                      workspace, stream)
+                      workspace, stream, kv_len_host)
+
+
+def hippo_verify_attention_layers_workspace_bytes(n_layers: int, batch: int, q_len: int, n_q_heads: int, n_kv_heads: int,
+                                                  head_dim: int) -> int:
+    return int(lib.hippo_verify_attention_layers_workspace_bytes(n_layers, batch, q_len, n_q_heads, n_kv_heads, head_dim))
+
+
+def hippo_verify_attention_layers(q_layers: Sequence[torch.Tensor], kv_layers: Sequence[KVCache], kv_len: Optional[torch.Tensor],
+                                  max_kv_len: int, out_layers: Sequence[torch.Tensor], softmax_scale: float = 0.0,
+                                  lse_layers: Optional[Sequence[Optional[torch.Tensor]]] = None,
+                                  workspace: Optional[torch.Tensor] = None, stream=None,
+                                  kv_len_host: Optional[Sequence[int]] = None):
+    """The verification attention of several layers in one launch: out_layers[l] = attention(q_layers[l], kv_layers[l])."""
+    n = len(q_layers)
+    assert n == len(kv_layers) == len(out_layers) and n > 0
+    B, q_len, hq, d = q_layers[0].shape
+    for q, o in zip(q_layers, out_layers):
+        assert q.is_contiguous() and o.is_contiguous() and q.shape == (B, q_len, hq, d) and o.shape == q.shape and o.dtype == q.dtype
+    assert kv_len is None or kv_len.dtype == torch.int32
+    if workspace is None:
+        workspace = new_workspace(hippo_verify_attention_layers_workspace_bytes(n, B, q_len, hq, kv_layers[0].n_kv_heads, d),
+                                  q_layers[0].device)
+    qp = (_vp * n)(*[t.data_ptr() for t in q_layers])
+    op = (_vp * n)(*[t.data_ptr() for t in out_layers])
+    lp = None
+    if lse_layers is not None:
+        lp = (_vp * n)(*[None if t is None else t.data_ptr() for t in lse_layers])
+    kvs = (KVCacheStruct * n)(*[c.struct for c in kv_layers])
+    _check(lib.hippo_verify_attention_layers(n, B, q_len, hq, qp, kvs, _ptr(kv_len),
+                                             None if kv_len_host is None else _host_i32(kv_len_host), int(max_kv_len),
+                                             float(softmax_scale), op, lp, _ptr(workspace), workspace.numel(), _stream(stream)))
+    return out_layers
 
 
 # ---- global semantic relevance (Eq. 2) ----------------------------------------------------------------------------
@@ -359,9 +436,10 @@ def hippo_accept(target_logits: torch.Tensor, draft_logits: Optional[torch.Tenso
     return n_accepted, out_tokens
 
 
-def hippo_accept_noalloc(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
-                         u_accept: torch.Tensor, u_resample: torch.Tensor, n_accepted: torch.Tensor,
-                         out_tokens: torch.Tensor, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+def hippo_accept_noalloc(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], draft_tokens: torch.Tensor,
+                         u_accept: Optional[torch.Tensor], u_resample: Optional[torch.Tensor], n_accepted: torch.Tensor,
+                         out_tokens: torch.Tensor, stream=None, mode: int = HIPPO_ACCEPT_SAMPLE
+                         ) -> Tuple[torch.Tensor, torch.Tensor]:
     """hippo_accept without a workspace argument, for callers that cannot allocate one (an engine that owns all
     device memory, a host that forbids cudaMalloc in its decode loop).  The scratch is a fixed array inside the
     library, shared by every call on the device; the outputs must be passed in because this wrapper allocates
@@ -370,11 +448,11 @@ def hippo_accept_noalloc(target_logits: torch.Tensor, draft_logits: torch.Tensor
     B, g1, V = target_logits.shape
     g = g1 - 1
     for t in (target_logits, draft_logits, u_accept, u_resample):
-        assert t.dtype == torch.float32 and t.is_contiguous()
+        assert t is None or (t.dtype == torch.float32 and t.is_contiguous())
     assert draft_tokens.dtype == torch.int32 and draft_tokens.is_contiguous()
     assert n_accepted.dtype == torch.int32 and n_accepted.numel() >= B
     assert out_tokens.dtype == torch.int32 and out_tokens.numel() >= B * (g + 1) and out_tokens.is_contiguous()
     _check(lib.hippo_accept_noalloc(B, g, V, _ptr(target_logits), _ptr(draft_logits) if g else None,
                                     _ptr(draft_tokens) if g else None, _ptr(u_accept) if g else None,
-                                    _ptr(u_resample), 0, _ptr(n_accepted), _ptr(out_tokens), _stream(stream)))
+                                    _ptr(u_resample), int(mode), _ptr(n_accepted), _ptr(out_tokens), _stream(stream)))
     return n_accepted, out_tokens

@@ -2,8 +2,13 @@
 
     one-time per prompt : hippo_select_tokens -> hippo_gather_kv (all draft layers in one launch)
     per decoding round  : stream D: gamma x n_draft_layers x hippo_draft_attention (q_len 1, pruned cache)
-                          stream V: n_target_layers x hippo_verify_attention (q_len gamma+1, full cache)
+                          stream V: the target layers' verification attention (q_len gamma+1, full cache), either
+                                    all layers in one hippo_verify_attention_layers call (default) or one
+                                    hippo_verify_attention call per layer
                           join -> hippo_accept
+
+In `run()` the verification stream is forked first: it reads neither the selection nor the gathered cache, so it
+runs beside select and gather as well as beside the draft calls.
 
 The draft and the verification kernels run on separate CUDA streams, mirroring the paper's decoupled
 draft/verify overlap (Section 5.2).  This module only allocates device memory through PyTorch, fills it with
@@ -28,8 +33,10 @@ def _randn(shape, dtype, gen, device):
 
 class HippoStep:
     def __init__(self, cfg: W.HippoConfig, device="cuda", target_layers: Optional[int] = None,
-                 draft_layers: Optional[int] = None, host_inputs: Optional[Dict[str, np.ndarray]] = None):
+                 draft_layers: Optional[int] = None, host_inputs: Optional[Dict[str, np.ndarray]] = None,
+                 multi_layer_verify: bool = True):
         self.cfg = cfg
+        self.multi_layer_verify = multi_layer_verify
         self.device = torch.device(device)
         self.Lt = cfg.tgt_layers if target_layers is None else target_layers
         self.Ld = cfg.dft_layers if draft_layers is None else draft_layers
@@ -97,6 +104,10 @@ class HippoStep:
         self.out_t = torch.empty_like(self.q_t)
         self.kv_len_t = torch.tensor(self.kv_len_t_host, dtype=torch.int32, device=self.device)
         self.verify_ws = hb.new_workspace(hb.hippo_attention_workspace_bytes(B, g + 1, cfg.tgt_q_heads, H, D), self.device)
+        self.verify_layers_ws = hb.new_workspace(
+            hb.hippo_verify_attention_layers_workspace_bytes(self.Lt, B, g + 1, cfg.tgt_q_heads, H, D), self.device)
+        self.q_t_layers = [self.q_t[l] for l in range(self.Lt)]
+        self.out_t_layers = [self.out_t[l] for l in range(self.Lt)]
 
         # ---- acceptance inputs (host-generated: the draft tokens are sampled from the draft logits)
         acc = W.accept_inputs(cfg) if host_inputs is None else host_inputs
@@ -129,6 +140,23 @@ class HippoStep:
     def select_bytes(self) -> int:
         return sum(self.n_visual) * self.cfg.embed_dim * self.elem
 
+    def select_flops(self) -> int:
+        """fp64 flops of the selection scores as defined (2 per multiply-add): per crop of M tokens M(M-1)/2 distinct
+        cosine dot products, per token one norm and one dot product with the same cell of the next frame."""
+        c = self.cfg
+        tpf = c.grid_h * c.grid_w
+        dots = 0
+        for n in self.n_visual:
+            full, rest = divmod(n, tpf)
+            for nf, count in ((tpf, full), (rest, 1 if rest else 0)):
+                for y0 in range(0, c.grid_h, c.crop_h):
+                    for x0 in range(0, c.grid_w, c.crop_w):
+                        m = sum(1 for y in range(y0, min(y0 + c.crop_h, c.grid_h)) for x in range(x0, min(x0 + c.crop_w, c.grid_w))
+                                if y * c.grid_w + x < nf)
+                        dots += count * m * (m - 1) // 2
+            dots += n + max(0, n - tpf)       # norms, and one temporal dot product per token that has a next frame
+        return 2 * dots * c.embed_dim
+
     def accept_bytes(self) -> int:
         c = self.cfg
         return c.batch * (2 * c.gamma + 1) * c.vocab * 4
@@ -139,6 +167,23 @@ class HippoStep:
         hb.hippo_select_tokens(self.embeds, self.attn_mass, self.n_visual, self.k, c.grid_h, c.grid_w, c.crop_h, c.crop_w,
                                kept_idx=self.keep_idx, kept_offsets=self.kept_offsets_host, fused_score=self.fused,
                                workspace=self.select_ws, stream=stream)
+
+    def select_with(self, **kw):
+        """hippo_select_tokens on this step's inputs with other options (score mask, policy); returns (kept, fused)."""
+        c = self.cfg
+        return hb.hippo_select_tokens(self.embeds, self.attn_mass, self.n_visual, self.k, c.grid_h, c.grid_w, c.crop_h,
+                                      c.crop_w, **kw)
+
+    def policy_variants(self):
+        """Named option sets of the selection whose kept sets the benchmark compares."""
+        gen = torch.Generator(device=self.device)
+        gen.manual_seed(4000 + self.cfg.seed)
+        keys = torch.rand(sum(self.n_visual), generator=gen, device=self.device, dtype=torch.float32)
+        return {"attention_only": {"score_mask": 1}, "all_terms": {"score_mask": 7},
+                "uniform_per_frame_attention_only": {"score_mask": 1, "policy": hb.HIPPO_SELECT_UNIFORM_PER_FRAME},
+                "uniform_per_frame_all_terms": {"score_mask": 7, "policy": hb.HIPPO_SELECT_UNIFORM_PER_FRAME},
+                "random": {"policy": hb.HIPPO_SELECT_RANDOM, "random_keys": keys},
+                "whole_frames": {"policy": hb.HIPPO_SELECT_FRAMES}}
 
     def gather(self, stream=None):
         hb.hippo_gather_kv(self.Ld, self.src_cache[0], self.src_layer_stride, self.dst_cache[0], self.dst_layer_stride,
@@ -151,10 +196,20 @@ class HippoStep:
                                          out=self.out_d[l, j], workspace=self.draft_ws, stream=stream)
 
     def verify(self, stream=None):
+        """The verification leg, one call per target layer."""
         m = max(self.kv_len_t_host)
         for l in range(self.Lt):
             hb.hippo_verify_attention(self.q_t[l], self.tgt_cache[l], self.kv_len_t, m, out=self.out_t[l],
-                                      workspace=self.verify_ws, stream=stream)
+                                      workspace=self.verify_ws, stream=stream, kv_len_host=self.kv_len_t_host)
+
+    def verify_layers(self, stream=None):
+        """The verification leg, all target layers in one call."""
+        hb.hippo_verify_attention_layers(self.q_t_layers, self.tgt_cache, self.kv_len_t, max(self.kv_len_t_host),
+                                         self.out_t_layers, workspace=self.verify_layers_ws, stream=stream,
+                                         kv_len_host=self.kv_len_t_host)
+
+    def verify_leg(self, stream=None):
+        (self.verify_layers if self.multi_layer_verify else self.verify)(stream)
 
     def attention_mass(self, stream=None):
         """Eq. 2 over all target layers of the prefilled cache (once per prompt, upstream of select); the result goes
@@ -189,12 +244,12 @@ class HippoStep:
     def run(self):
         """The whole step on the current stream, with draft and verify forked onto their own streams."""
         main = torch.cuda.current_stream(self.device)
+        self.stream_v.wait_stream(main)
+        self.verify_leg(self.stream_v)        # reads neither the selection nor the pruned cache
         self.select(main)
         self.gather(main)
         self.stream_d.wait_stream(main)
-        self.stream_v.wait_stream(main)
-        self.draft(self.stream_d)
-        self.verify(self.stream_v)
+        self.draft(self.stream_d)             # reads the gathered cache
         main.wait_stream(self.stream_d)
         main.wait_stream(self.stream_v)
         self.accept(main)

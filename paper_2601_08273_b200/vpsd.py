@@ -40,8 +40,8 @@ class VpsdLoop:
         self.q_t = _randn((st.Lt, 1, mb + 1, cfg.tgt_q_heads, cfg.tgt_head_dim), st.tdt, gen, self.dev)
         self.out_t = torch.empty_like(self.q_t)
         self.kv_len_t = {c: torch.tensor([st.ctx[0] + c + 1], dtype=torch.int32, device=self.dev) for c in range(1, mb + 1)}
-        self.verify_ws = hb.new_workspace(hb.hippo_attention_workspace_bytes(1, mb + 1, cfg.tgt_q_heads, cfg.tgt_kv_heads,
-                                                                             cfg.tgt_head_dim), self.dev)
+        self.verify_ws = hb.new_workspace(hb.hippo_verify_attention_layers_workspace_bytes(
+            st.Lt, 1, mb + 1, cfg.tgt_q_heads, cfg.tgt_kv_heads, cfg.tgt_head_dim), self.dev)
         # acceptance inputs: a pool of rounds; draft logits = target logits + noise, draft tokens drawn from them
         V = cfg.vocab
         self.pool = []
@@ -57,9 +57,9 @@ class VpsdLoop:
         self.out_tokens = torch.empty((1, mb + 1), dtype=torch.int32, device=self.dev)
         self.accept_ws = hb.new_workspace(hb.hippo_accept_workspace_bytes(1, mb, V), self.dev)
         self.stream_d, self.stream_v = st.stream_d, st.stream_v
-        # One draft token (draft_layers launches) and one verification pass (target_layers launches) are launch-bound
-        # when issued call by call from one host thread, which would serialise the two streams on the host: each is
-        # captured once into a CUDA graph and replayed.
+        # One draft token (draft_layers launches) is launch-bound when issued call by call from one host thread, which
+        # would serialise the two streams on the host: it is captured once into a CUDA graph and replayed, and so is the
+        # verification pass of each batch size.
         self.g_draft = {}
         self.g_verify = {}
         if use_graphs:
@@ -89,9 +89,10 @@ class VpsdLoop:
 
     def _verify_eager(self, c: int, stream) -> None:
         st = self.st
-        for l in range(st.Lt):
-            hb.hippo_verify_attention(self.q_t[l][:, :c + 1], st.tgt_cache[l], self.kv_len_t[c], st.ctx[0] + c + 1,
-                                      out=self.out_t[l][:, :c + 1], workspace=self.verify_ws, stream=stream)
+        # the verification pass: every target layer's attention in one launch
+        hb.hippo_verify_attention_layers([self.q_t[l][:, :c + 1] for l in range(st.Lt)], st.tgt_cache, self.kv_len_t[c],
+                                         st.ctx[0] + c + 1, [self.out_t[l][:, :c + 1] for l in range(st.Lt)],
+                                         workspace=self.verify_ws, stream=stream, kv_len_host=[st.ctx[0] + c + 1])
 
     def draft_token(self, j: int, stream) -> None:
         jj = j % self.cfg.gamma

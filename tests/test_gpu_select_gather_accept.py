@@ -114,6 +114,84 @@ def test_c4_select_whole_sequence(hb):
         check_kept(host(kept), host(fused), ref_idx, ref_fused, kth, "c4 keep %d%%" % pct)
 
 
+# ---- the other selection rules ------------------------------------------------------------------------------------
+
+def check_kept_per_frame(got_idx, ref_fused, k, tpf, what):
+    """Uniform per-frame budget: per frame the kept sets agree except for tokens whose oracle score lies within 1e-6
+    (relative) of that frame's own threshold; the budgets agree exactly."""
+    ref_idx, budget = oracle.select_policy(oracle.POLICY_UNIFORM_PER_FRAME, ref_fused, k, tpf)
+    assert len(got_idx) == k and np.all(np.diff(got_idx) > 0), what
+    assert np.bincount(got_idx // tpf, minlength=len(budget)).tolist() == budget.tolist(), what + ": per-frame counts"
+    diff = np.setxor1d(got_idx, ref_idx)
+    for j in diff:
+        f = j // tpf
+        kth = np.sort(ref_fused[f * tpf:(f + 1) * tpf])[::-1][budget[f] - 1]
+        assert abs(ref_fused[j] - kth) <= 1e-6 * abs(kth), "%s: token %d differs outside the near-tie band of frame %d" % (what, j, f)
+
+
+@pytest.mark.parametrize("ci,mask", [(0, 7), (0, 1), (1, 7), (1, 1)])
+def test_select_uniform_per_frame(hb, ci, mask):
+    cfg = W.CONFIGS[ci]
+    inp = W.select_inputs(cfg)
+    E, m = dev(inp["embeds"], cfg.dtype), dev(inp["attn_mass"])
+    ref_fused, _, _ = oracle.select_scores(inp["embeds"], inp["attn_mass"], cfg.grid_h, cfg.grid_w, score_mask=mask)
+    for k in (inp["k"], 0, 1, cfg.frames - 1, inp["n_visual"] - 3, inp["n_visual"]):
+        kept, fused = hb.hippo_select_tokens(E, m, [inp["n_visual"]], [k], cfg.grid_h, cfg.grid_w, score_mask=mask,
+                                             policy=hb.HIPPO_SELECT_UNIFORM_PER_FRAME)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(host(fused), ref_fused, rtol=0, atol=2e-6)
+        check_kept_per_frame(host(kept), ref_fused, k, cfg.tokens_per_frame, "c%d mask %d k %d" % (ci, mask, k))
+
+
+def test_select_policies_ragged_batch_with_partial_frames(hb):
+    """Four sequences, three with a partial last frame (one of them a single frame of 9 tokens): per-frame budgets with
+    a shortfall, random keys, whole frames; kept lists written at explicit offsets."""
+    cfg = W.CONFIGS[3].replace(embed_dim=128)
+    tpf = cfg.tokens_per_frame
+    lens = [tpf * 3 + 57, tpf * 2, tpf + 1, 9]
+    embeds = [W.select_inputs(cfg, b, n)["embeds"] for b, n in enumerate(lens)]
+    masses = [W.attention_mass(cfg, n, b) for b, n in enumerate(lens)]
+    E, m = dev(np.concatenate(embeds), "bf16"), dev(np.concatenate(masses))
+    rng = np.random.default_rng(5)
+    keys = rng.random(sum(lens)).astype(np.float32)
+    ks = [tpf * 2 + 100, 30, tpf, 4]            # sequence 0: 4 frames, the last (57 tokens) cannot take its 123
+    offs = [0, 1000, 2000, 3000]
+    starts = np.concatenate([[0], np.cumsum(lens)])
+    for policy in (hb.HIPPO_SELECT_UNIFORM_PER_FRAME, hb.HIPPO_SELECT_RANDOM, hb.HIPPO_SELECT_FRAMES):
+        kept = torch.full((3300,), -1, dtype=torch.int32, device="cuda")
+        _, fused = hb.hippo_select_tokens(E, m, lens, ks, 14, 14, policy=policy, random_keys=dev(keys) if policy == hb.HIPPO_SELECT_RANDOM else None,
+                                          kept_idx=kept, kept_offsets=offs)
+        torch.cuda.synchronize()
+        kept = host(kept)
+        for b, n in enumerate(lens):
+            got = kept[offs[b]:offs[b] + ks[b]]
+            if policy == hb.HIPPO_SELECT_UNIFORM_PER_FRAME:
+                ref_fused, _, _ = oracle.select_scores(embeds[b], masses[b], 14, 14)
+                check_kept_per_frame(got, ref_fused, ks[b], tpf, "seq %d" % b)
+            else:
+                score = keys[starts[b]:starts[b + 1]]
+                want, _ = oracle.select_policy(policy, score, ks[b], tpf)
+                assert got.tolist() == want.tolist(), "policy %d seq %d" % (policy, b)
+            assert np.all(kept[offs[b] + ks[b]:(offs[b + 1] if b + 1 < len(offs) else None)] == -1)   # nothing beyond k[b]
+        if policy == hb.HIPPO_SELECT_RANDOM:
+            np.testing.assert_array_equal(host(fused), keys)
+
+
+def test_select_random_and_frames_need_no_embeddings(hb):
+    cfg = W.CONFIGS[2]
+    n, tpf = W.visual_lengths(cfg)[0], cfg.tokens_per_frame
+    keys = np.random.default_rng(6).random(n).astype(np.float32)
+    keys[100:140] = keys[7]                                        # a run of equal keys across the threshold region
+    for k in (W.keep_count(n, 10), 1, n):
+        kept, _ = hb.hippo_select_tokens(None, None, [n], [k], cfg.grid_h, cfg.grid_w, policy=hb.HIPPO_SELECT_RANDOM, random_keys=dev(keys))
+        torch.cuda.synchronize()
+        assert host(kept).tolist() == oracle.select_policy(oracle.POLICY_RANDOM, keys, k, tpf)[0].tolist()
+    for k in (W.keep_count(n, 10), tpf * 13, 5, n - 1, n):
+        kept, _ = hb.hippo_select_tokens(None, None, [n], [k], cfg.grid_h, cfg.grid_w, policy=hb.HIPPO_SELECT_FRAMES)
+        torch.cuda.synchronize()
+        assert host(kept).tolist() == oracle.select_policy(oracle.POLICY_FRAME, np.zeros(n), k, tpf)[0].tolist()
+
+
 def test_topk_all_three_key_tiers(hb):
     """100,352 tokens: keys in registers, in shared memory and re-read from memory; many equal scores (attention term
     only, mass quantised to 64 levels) so that the index tie-break decides most of the threshold."""
@@ -188,6 +266,58 @@ def test_gather_config_shapes(hb, ci, keep_pct):
     run_gather(hb, cfg, 2, src_lens, keeps, cfg.dtype, shuffle=(3, 4) if cfg.paged_shuffle else (None, None))
 
 
+def test_gather_skips_out_of_range_entries_and_says_so(hb):
+    """A keep index beyond the source's pages, a negative one, a page id outside the pool and a sequence that keeps more
+    than its destination holds: nothing is read or written for those entries, the flag word is raised, every valid entry is
+    still copied."""
+    cfg = W.CONFIGS[0]
+    H, D = cfg.dft_kv_heads, cfg.dft_head_dim
+    rng = np.random.default_rng(3)
+    src_lens = [200, 100]
+    k = rng.standard_normal((2, 200, H, D)).astype(np.float32)
+    st, sp = W.make_page_table(src_lens, np.random.default_rng(1))
+    src_pool = dev(W.pack_paged(k, src_lens, st, sp))
+    src = hb.KVCache(src_pool, src_pool.clone(), dev(st))
+
+    def run(keeps, dst_table, n_dst_pages, src_cache=src):
+        dst_k = torch.full((n_dst_pages, H, 64, D), -7.0, dtype=torch.float32, device="cuda")
+        dst = hb.KVCache(dst_k, dst_k.clone(), dev(dst_table))
+        offs = np.concatenate([[0], np.cumsum([len(x) for x in keeps])]).astype(np.int32)
+        flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+        hb.hippo_gather_kv(1, src_cache, 0, dst, 0, len(keeps), dev(np.concatenate(keeps).astype(np.int32)), dev(offs),
+                           int(offs[-1]), bad_index=flag)
+        torch.cuda.synchronize()
+        return host(dst_k), int(flag.item())
+
+    dt, dp = W.make_page_table([64, 64], None)
+    good = [np.array([5, 17, 199]), np.array([0, 99])]
+    got, flag = run(good, dt, dp)
+    assert flag == 0
+    assert np.array_equal(got[dt[0, 0], :, :3], np.transpose(k[0, good[0]], (1, 0, 2)))
+    # one entry past the source's page capacity (4 pages = 256 positions), one negative
+    bad = [np.array([5, 256, 199]), np.array([-1, 99])]
+    got, flag = run(bad, dt, dp)
+    assert flag == 1
+    assert np.array_equal(got[dt[0, 0], :, 0], k[0, 5]) and np.array_equal(got[dt[0, 0], :, 2], k[0, 199])
+    assert np.all(got[dt[0, 0], :, 1] == -7.0) and np.all(got[dt[1, 0], :, 0] == -7.0)      # skipped: destination untouched
+    assert np.array_equal(got[dt[1, 0], :, 1], k[1, 99])
+    # a page id outside the source pool
+    st_bad = st.copy()
+    st_bad[0, 0] = sp + 5
+    got, flag = run(good, dt, dp, hb.KVCache(src_pool, src_pool.clone(), dev(st_bad)))
+    assert flag == 1 and np.all(got[dt[0, 0], :, :2] == -7.0) and np.array_equal(got[dt[0, 0], :, 2], k[0, 199])
+    # sequence 0 keeps 70 tokens but its destination row holds one page: entries 64.. are skipped, not spilled into sequence 1
+    many = [np.arange(70), np.array([3])]
+    got, flag = run(many, dt, dp)
+    assert flag == 1
+    assert np.array_equal(got[dt[0, 0]], np.transpose(k[0, :64], (1, 0, 2)))
+    assert np.array_equal(got[dt[1, 0], :, 0], k[1, 3]) and np.all(got[dt[1, 0], :, 1:] == -7.0)
+    # more entries than the destination can hold at all: refused on the host
+    with pytest.raises(hb.HippoError) as e:
+        run([np.arange(100), np.arange(100)], dt, dp)
+    assert e.value.status == hb.HIPPO_ERR_INVALID_ARG
+
+
 # ---- acceptance -----------------------------------------------------------------------------------------------------
 
 def check_accept(hb, inp, what, forgiven_allowed=0):
@@ -239,6 +369,26 @@ def test_accept_odd_vocab_and_gamma0(hb):
     check_accept(hb, W.accept_inputs(cfg, batch=5, gamma=3, vocab=4099, corr_eps=0.5), "V=4099")
     check_accept(hb, W.accept_inputs(cfg, batch=3, gamma=0, vocab=777), "gamma 0")
     check_accept(hb, W.accept_inputs(cfg, batch=3, gamma=1, vocab=3, corr_eps=2.0), "V=3")
+
+
+def test_accept_draft_token_outside_the_vocabulary_is_rejected(hb):
+    """A draft token id that is not in [0, vocab) is never used as an index: it counts as rejected and the replacement is
+    drawn from the residual of its row, exactly as the oracle does for a token whose acceptance test fails."""
+    cfg = W.CONFIGS[0]
+    inp = W.accept_inputs(cfg, batch=6, gamma=4, vocab=777, corr_eps=0.0)       # draft == target: all accepted otherwise
+    x = inp["draft_tokens"].copy()
+    x[1, 2], x[2, 0], x[4, 3] = 777, -5, 1 << 30
+    n, out = hb.hippo_accept(dev(inp["target_logits"]), dev(inp["draft_logits"]), dev(x), dev(inp["u_accept"]),
+                             dev(inp["u_resample"]))
+    torch.cuda.synchronize()
+    n, out = host(n), host(out)
+    assert n.tolist() == [4, 2, 0, 4, 3, 4]
+    for b, j in ((1, 2), (2, 0), (4, 3)):
+        assert out[b, :j].tolist() == x[b, :j].tolist() and 0 <= out[b, j] < 777 and (out[b, j + 1:] == -1).all()
+    # the untouched sequences still match the oracle
+    rn, rout, _, _ = oracle.accept(inp["target_logits"], inp["draft_logits"], inp["draft_tokens"], inp["u_accept"], inp["u_resample"])
+    for b in (0, 3, 5):
+        assert n[b] == rn[b] and out[b].tolist() == rout[b].tolist()
 
 
 @pytest.mark.parametrize("ci", [0, 1, 3])

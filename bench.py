@@ -311,11 +311,13 @@ def kernel_sweep(cfg, torch, hb, HippoStep, peaks, uuid, reps=20, max_gb=24.0, b
     return out
 
 
-def schedule_entry(cfg, torch, hb, rounds=40):
-    """The adaptive decoding schedule (Section 5.2) over the kernels against the serial schedule."""
+def schedule_entry(cfg, torch, hb, rounds=40, draft_noise=0.5, verify_max_ctas=0):
+    """The adaptive decoding schedule (Section 5.2) over the kernels against the serial schedule.  draft_noise sets how far
+    the synthetic draft logits are from the target's (the acceptance rate); verify_max_ctas > 0 leaves SMs to the draft
+    stream while the verification kernel runs."""
     from paper_2601_08273_b200.vpsd import VpsdLoop
     torch.cuda.empty_cache()
-    loop = VpsdLoop(cfg, buffered=0, pool=8, draft_noise=0.5)
+    loop = VpsdLoop(cfg, buffered=0, pool=8, draft_noise=draft_noise, verify_max_ctas=verify_max_ctas)
     unit = loop.unit_times_ms()
     loop.run(4); loop.run_serial(2)
     par, ser = loop.run(rounds), loop.run_serial(rounds // 2)
@@ -327,6 +329,7 @@ def schedule_entry(cfg, torch, hb, rounds=40):
         hb.hippo_vpsd_commit(state, rd, t["accepted"], t["drafted_during"])
     serial_model = sum(hb.hippo_vpsd_serial_round_time(cfg.gamma, unit["t_draft"], unit["t_target"]) for _ in range(ser["rounds"]))
     out = {"workload": cfg.name + " decoding schedule", "gamma": cfg.gamma, "rounds": par["rounds"],
+           "draft_noise": draft_noise, "verify_max_ctas": verify_max_ctas,
            "t_draft_token_ms": round(unit["t_draft"], 4), "t_verify_ms": round(unit["t_target"], 4),
            "target_over_draft": round(unit["t_target"] / unit["t_draft"], 2),
            "parallel_tokens": par["tokens"], "parallel_ms": round(par["wall_ms"], 3),
@@ -542,11 +545,14 @@ def run_ours(args):
             del stb
         except Exception as e:  # noqa: BLE001
             extra.append({"workload": cfg.name + " kept-token border share", "error": str(e)[:200]})
+        # at two acceptance rates (a draft far from / close to the target), with all SMs for the verification kernel and
+        # with 32 of them left to the draft stream
         for ci in (1, 2, 4):
-            try:
-                extra.append(schedule_entry(W.CONFIGS[ci], torch, hb))
-            except Exception as e:  # noqa: BLE001
-                extra.append({"workload": W.CONFIGS[ci].name + " decoding schedule", "error": str(e)[:200]})
+            for noise, ctas in ((0.5, 0), (0.1, 0), (0.1, 116)):
+                try:
+                    extra.append(schedule_entry(W.CONFIGS[ci], torch, hb, draft_noise=noise, verify_max_ctas=ctas))
+                except Exception as e:  # noqa: BLE001
+                    extra.append({"workload": W.CONFIGS[ci].name + " decoding schedule", "error": str(e)[:200]})
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

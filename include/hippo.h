@@ -52,6 +52,10 @@ typedef enum hippo_status {
 typedef enum hippo_dtype { HIPPO_DTYPE_FP32 = 0, HIPPO_DTYPE_BF16 = 1 } hippo_dtype_t;
 
 typedef enum hippo_accept_mode { HIPPO_ACCEPT_SAMPLE = 0, HIPPO_ACCEPT_GREEDY = 1 } hippo_accept_mode_t;
+/* optional flags OR-ed into the mode of the sampling acceptance: force one of its two launch forms (same arithmetic, same
+ * results; without a flag the library picks the faster one for the shape) */
+#define HIPPO_ACCEPT_ONE_LAUNCH 16      /* one kernel, its CTAs meet at two counters in the workspace header */
+#define HIPPO_ACCEPT_THREE_LAUNCHES 32  /* three chained kernels */
 
 /* selection rules of hippo_select_tokens_policy */
 typedef enum hippo_select_policy {
@@ -263,6 +267,9 @@ int32_t hippo_draft_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, c
  *   kv_layers              HOST array [n_layers] of descriptors
  *   lse_layers             NULL, or HOST array [n_layers] of DEVICE pointers (entries may be NULL)
  *   kv_len, kv_len_host, max_kv_len, softmax_scale   as for hippo_verify_attention
+ *   max_ctas               0: one CTA per SM.  Otherwise an upper bound of the grid: the launch holds its SMs (all of their
+ *                          shared memory) from the first layer to the last, so a caller that wants kernels of another
+ *                          stream to run beside it - the draft model's, Section 5.2 - leaves them some SMs this way
  * The host arrays are read before the call returns.  The call enqueues one memset of its counters and one kernel
  * per 64 layers.  The workspace is larger than a single-layer one (three sets of partial-result slots and per-layer
  * counters): size it with hippo_verify_attention_layers_workspace_bytes.  bf16 with head_dim 64 or 128 and at most
@@ -275,7 +282,7 @@ size_t hippo_verify_attention_layers_workspace_bytes(int32_t n_layers, int32_t b
 int32_t hippo_verify_attention_layers(int32_t n_layers, int32_t batch, int32_t q_len, int32_t n_q_heads,
                                       const void *const *q_layers, const hippo_kv_cache_t *kv_layers,
                                       const int32_t *kv_len, const int32_t *kv_len_host, int32_t max_kv_len,
-                                      float softmax_scale, void *const *out_layers, float *const *lse_layers,
+                                      float softmax_scale, int32_t max_ctas, void *const *out_layers, float *const *lse_layers,
                                       void *workspace, size_t workspace_bytes, void *stream);
 
 /* ---- acceptance: Section 3.2, Eq. 1 -------------------------------------------------------------------------- */

@@ -36,6 +36,8 @@ HIPPO_SCORE_ALL = 7
 HIPPO_SELECT_HOLISTIC, HIPPO_SELECT_UNIFORM_PER_FRAME, HIPPO_SELECT_RANDOM, HIPPO_SELECT_FRAMES = 0, 1, 2, 3
 HIPPO_ACCEPT_SAMPLE = 0
 HIPPO_ACCEPT_GREEDY = 1
+HIPPO_ACCEPT_ONE_LAUNCH = 16
+HIPPO_ACCEPT_THREE_LAUNCHES = 32
 PAGE_SIZE = 64
 
 _vp, _i32, _u32, _sz, _f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_float
@@ -79,7 +81,7 @@ for _name in ("hippo_verify_attention", "hippo_draft_attention"):
 lib.hippo_verify_attention_layers_workspace_bytes.restype = _sz
 lib.hippo_verify_attention_layers_workspace_bytes.argtypes = [_i32] * 6
 lib.hippo_verify_attention_layers.restype = _i32
-lib.hippo_verify_attention_layers.argtypes = [_i32, _i32, _i32, _i32, ctypes.POINTER(_vp), _KVP, _vp, _I32P, _i32, _f32,
+lib.hippo_verify_attention_layers.argtypes = [_i32, _i32, _i32, _i32, ctypes.POINTER(_vp), _KVP, _vp, _I32P, _i32, _f32, _i32,
                                               ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, _sz, _vp]
 lib.hippo_workspace_set_wait_limit.restype = _i32
 lib.hippo_workspace_set_wait_limit.argtypes = [_vp, ctypes.c_int64, _vp]
@@ -325,8 +327,9 @@ def hippo_verify_attention_layers(q_layers: Sequence[torch.Tensor], kv_layers: S
                                   max_kv_len: int, out_layers: Sequence[torch.Tensor], softmax_scale: float = 0.0,
                                   lse_layers: Optional[Sequence[Optional[torch.Tensor]]] = None,
                                   workspace: Optional[torch.Tensor] = None, stream=None,
-                                  kv_len_host: Optional[Sequence[int]] = None):
-    """The verification attention of several layers in one launch: out_layers[l] = attention(q_layers[l], kv_layers[l])."""
+                                  kv_len_host: Optional[Sequence[int]] = None, max_ctas: int = 0):
+    """The verification attention of several layers in one launch: out_layers[l] = attention(q_layers[l], kv_layers[l]).
+    max_ctas > 0 bounds the grid, leaving the other SMs to kernels of other streams."""
     n = len(q_layers)
     assert n == len(kv_layers) == len(out_layers) and n > 0
     B, q_len, hq, d = q_layers[0].shape
@@ -344,7 +347,8 @@ def hippo_verify_attention_layers(q_layers: Sequence[torch.Tensor], kv_layers: S
     kvs = (KVCacheStruct * n)(*[c.struct for c in kv_layers])
     _check(lib.hippo_verify_attention_layers(n, B, q_len, hq, qp, kvs, _ptr(kv_len),
                                              None if kv_len_host is None else _host_i32(kv_len_host), int(max_kv_len),
-                                             float(softmax_scale), op, lp, _ptr(workspace), workspace.numel(), _stream(stream)))
+                                             float(softmax_scale), int(max_ctas), op, lp, _ptr(workspace), workspace.numel(),
+                                             _stream(stream)))
     return out_layers
 
 

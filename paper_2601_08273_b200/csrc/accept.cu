@@ -16,6 +16,7 @@
 //           u * total; only that one group's weights are evaluated again
 #include <math.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -26,6 +27,7 @@ constexpr int kAccThreads = 256;
 constexpr int kAccPerThread = 16;
 constexpr int kAccChunk = kAccThreads * kAccPerThread;  // 4096 vocabulary entries per chunk
 constexpr int kAccMaxRows = 2 * 64 + 1;
+constexpr bool kAcceptFusedByDefault = false;
 
 struct RowInfo {
     double Mp, Zp, Mq, Zq;  // max logit and 1 / (sum of exponentials) of target row n / draft row n
@@ -72,12 +74,12 @@ __device__ double block_scan_inclusive(double v, double *warp_tot /* [8] shared 
     return v + pre;
 }
 
-__global__ void __launch_bounds__(kAccThreads) accept_stats_kernel(const AcceptParams p) {
+// Max and sum of exponentials of one 4096-token chunk of one logit row.
+__device__ void stats_item(const AcceptParams &p, int b, int r, int c) {
     __shared__ float smax[kAccThreads / 32];
     __shared__ double ssum[kAccThreads / 32];
-    pdl_wait();
-    pdl_trigger();
-    const int c = blockIdx.x, r = blockIdx.y, b = blockIdx.z, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __syncthreads();   // the shared arrays may still be read by the previous item
     const float *row = logit_row(p, b, r);
     float v[kAccPerThread];
     float m = -INFINITY;
@@ -114,6 +116,12 @@ __global__ void __launch_bounds__(kAccThreads) accept_stats_kernel(const AcceptP
         for (int w = 0; w < kAccThreads / 32; ++w) tot += ssum[w];
         p.stats[((size_t)b * (2 * p.gamma + 1) + r) * p.n_chunks + c] = make_double2((double)m, tot);
     }
+}
+
+__global__ void __launch_bounds__(kAccThreads) accept_stats_kernel(const AcceptParams p) {
+    pdl_wait();
+    pdl_trigger();
+    stats_item(p, blockIdx.z, blockIdx.y, blockIdx.x);
 }
 
 // Weight of token t in the distribution the emitted token is drawn from.  use_target_only: bonus row, or the
@@ -212,19 +220,20 @@ __device__ RowInfo decide_rows(const AcceptParams &p, int b, double *rowstat /* 
     return ri;
 }
 
-__global__ void __launch_bounds__(kAccThreads) accept_weigh_kernel(const AcceptParams p) {
+// Residual (or bonus) weights of one chunk of sequence b, scanned in token order.  Every caller re-derives the row
+// normalisers and the accept decisions of the sequence (same data, same order: identical everywhere).
+__device__ void weigh_item(const AcceptParams &p, int b, int c) {
     __shared__ double rowstat[2 * kAccMaxRows];
     __shared__ double warp_tot[kAccThreads / 32];
     __shared__ int s_n;
-    pdl_wait();
-    pdl_trigger();
-    const int c = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const int tid = threadIdx.x;
+    __syncthreads();   // the shared arrays may still be read by the previous item
     const RowInfo ri = decide_rows(p, b, rowstat, &s_n);
     if (c == 0 && tid == 0) {
         const int32_t *x = p.x + (size_t)b * p.gamma;
         int32_t *out = p.out + (size_t)b * (p.gamma + 1);
         for (int j = 0; j < ri.n; ++j) out[j] = x[j];
-        for (int j = ri.n; j <= p.gamma; ++j) out[j] = -1;  // out[n] is filled by the pick kernel
+        for (int j = ri.n; j <= p.gamma; ++j) out[j] = -1;  // out[n] is filled by the pick step
         p.n_acc[b] = ri.n;
         p.info[b] = ri;
     }
@@ -237,14 +246,20 @@ __global__ void __launch_bounds__(kAccThreads) accept_weigh_kernel(const AcceptP
     if (tid == 0) p.wsum[(size_t)b * p.n_chunks + c] = total;
 }
 
-__global__ void __launch_bounds__(kAccThreads) accept_pick_kernel(const AcceptParams p) {
+__global__ void __launch_bounds__(kAccThreads) accept_weigh_kernel(const AcceptParams p) {
+    pdl_wait();
+    pdl_trigger();
+    weigh_item(p, blockIdx.y, blockIdx.x);
+}
+
+// The emitted token of sequence b: chunk, 16-token group and token where the CDF crosses u * total.  ws: n_chunks doubles of
+// shared memory.
+__device__ void pick_item(const AcceptParams &p, int b, double *ws) {
     __shared__ double warp_tot[kAccThreads / 32];
     __shared__ double s_prefix, s_target;
     __shared__ int s_chunk, s_tok, s_target_only;
-    extern __shared__ double ws[];   // [n_chunks] chunk weights
-    pdl_wait();
-    pdl_trigger();
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int tid = threadIdx.x;
+    __syncthreads();   // the shared arrays may still be read by the previous item
     const RowInfo ri = p.info[b];
     const float *trow = logit_row(p, b, ri.n);
     const float *drow = ri.bonus ? nullptr : logit_row(p, b, p.gamma + 1 + ri.n);
@@ -342,6 +357,62 @@ __global__ void __launch_bounds__(kAccThreads) accept_pick_kernel(const AcceptPa
     if (tid == 0) p.out[(size_t)b * (p.gamma + 1) + ri.n] = tok;
 }
 
+__global__ void __launch_bounds__(kAccThreads) accept_pick_kernel(const AcceptParams p) {
+    extern __shared__ double ws[];   // [n_chunks] chunk weights
+    pdl_wait();
+    pdl_trigger();
+    pick_item(p, blockIdx.x, ws);
+}
+
+// ---- the same three steps in one launch ----------------------------------------------------------------------------
+// A grid of at most one wave of CTAs walks the items of each step; between the steps all CTAs meet at a counter in the
+// workspace header (zeroed before the launch).  The wait at the counter is bounded: after 2 s a CTA records
+// HIPPO_ERR_TIMEOUT in the header and leaves, and so does every CTA that sees the status word set.
+constexpr unsigned long long kAccWaitLimitNs = 2000000000ull;
+
+__device__ bool accept_grid_barrier(WsHeader *hdr, int which) {
+    __shared__ int s_ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int *counter = &hdr->pad[which];
+        __threadfence();
+        atomicAdd(counter, 1);
+        bool ok = true;
+        unsigned long long t0 = 0;
+        for (;;) {
+            int seen;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+            if (seen >= (int)gridDim.x) break;
+            if (*reinterpret_cast<volatile int *>(&hdr->status) != 0) { ok = false; break; }
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kAccWaitLimitNs) {
+                if (atomicCAS(&hdr->status, 0, (int)HIPPO_ERR_TIMEOUT) == 0) hdr->where = 200 + which;
+                ok = false;
+                break;
+            }
+            __nanosleep(64);
+        }
+        s_ok = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return s_ok != 0;
+}
+
+__global__ void __launch_bounds__(kAccThreads) accept_fused_kernel(const AcceptParams p, WsHeader *hdr) {
+    extern __shared__ double ws[];   // [n_chunks] chunk weights
+    pdl_wait();
+    pdl_trigger();
+    const int rows = 2 * p.gamma + 1;
+    for (int i = blockIdx.x; i < p.B * rows * p.n_chunks; i += gridDim.x)
+        stats_item(p, i / (rows * p.n_chunks), (i / p.n_chunks) % rows, i % p.n_chunks);
+    if (!accept_grid_barrier(hdr, 0)) return;
+    for (int i = blockIdx.x; i < p.B * p.n_chunks; i += gridDim.x) weigh_item(p, i / p.n_chunks, i % p.n_chunks);
+    if (!accept_grid_barrier(hdr, 1)) return;
+    for (int b = blockIdx.x; b < p.B; b += gridDim.x) pick_item(p, b, ws);
+}
+
 struct AcceptWs { size_t stats_off, wsum_off, info_off, tscan_off, total; int n_chunks; };
 static AcceptWs accept_ws(int B, int gamma, int V) {
     AcceptWs w;
@@ -434,7 +505,7 @@ static int32_t launch_accept_greedy(const AcceptParams &p, cudaStream_t s) {
 }
 
 // The three kernels, launched with programmatic stream serialization (each one waits before it reads).
-static int32_t launch_accept(const AcceptParams &p, cudaStream_t s) {
+static int32_t launch_accept_chain(const AcceptParams &p, cudaStream_t s) {
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -454,6 +525,47 @@ static int32_t launch_accept(const AcceptParams &p, cudaStream_t s) {
     return HIPPO_OK;
 }
 
+// One launch: the grid is at most what the device keeps resident at once (the CTAs wait for one another between the
+// steps), and never more than the first step has items.
+static int32_t launch_accept_fused(const AcceptParams &p, WsHeader *hdr, cudaStream_t s) {
+    const size_t smem = (size_t)p.n_chunks * sizeof(double);
+    if (smem > 40 * 1024) return launch_accept_chain(p, s);
+    static std::atomic<int> resident[kMaxDevices];
+    int dev = -1;
+    HIPPO_CUDA_TRY(cudaGetDevice(&dev));
+    int cap = (dev >= 0 && dev < kMaxDevices) ? resident[dev].load(std::memory_order_relaxed) : 0;
+    if (cap == 0) {
+        int per_sm = 0, sms = 0;
+        HIPPO_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, accept_fused_kernel, kAccThreads, 40 * 1024));
+        HIPPO_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        cap = per_sm * sms;
+        if (cap < 1) return launch_accept_chain(p, s);
+        if (dev >= 0 && dev < kMaxDevices) resident[dev].store(cap, std::memory_order_relaxed);
+    }
+    long long grid = (long long)p.B * (2 * p.gamma + 1) * p.n_chunks;
+    if (grid > cap) grid = cap;
+    HIPPO_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s));    // status word and the two arrival counters
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kAccThreads);
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    HIPPO_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_fused_kernel, p, hdr));
+    count_launches(1);
+    return HIPPO_OK;
+}
+
+// variant: 0 the faster of the two for the shape, else HIPPO_ACCEPT_ONE_LAUNCH / HIPPO_ACCEPT_THREE_LAUNCHES
+static int32_t launch_accept(const AcceptParams &p, WsHeader *hdr, int variant, cudaStream_t s) {
+    const bool fused = variant == HIPPO_ACCEPT_ONE_LAUNCH || (variant == 0 && kAcceptFusedByDefault);
+    return fused ? launch_accept_fused(p, hdr, s) : launch_accept_chain(p, s);
+}
+
 }  // namespace hippo
 
 extern "C" {
@@ -469,7 +581,10 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
                      void *workspace, size_t workspace_bytes, void *stream) {
     using namespace hippo;
     if (batch <= 0 || gamma < 0 || vocab <= 0) return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept: bad sizes");
-    if (mode != HIPPO_ACCEPT_SAMPLE && mode != HIPPO_ACCEPT_GREEDY) return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept: mode %d", mode);
+    const int variant = mode & (HIPPO_ACCEPT_ONE_LAUNCH | HIPPO_ACCEPT_THREE_LAUNCHES);
+    mode &= ~(HIPPO_ACCEPT_ONE_LAUNCH | HIPPO_ACCEPT_THREE_LAUNCHES);
+    if ((mode != HIPPO_ACCEPT_SAMPLE && mode != HIPPO_ACCEPT_GREEDY) || variant == (HIPPO_ACCEPT_ONE_LAUNCH | HIPPO_ACCEPT_THREE_LAUNCHES))
+        return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept: mode %d", mode | variant);
     const bool greedy = mode == HIPPO_ACCEPT_GREEDY;
     if (!target_logits || !n_accepted || !out_tokens || !workspace || (!greedy && !u_resample))
         return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept: null pointer");
@@ -490,7 +605,7 @@ int32_t hippo_accept(int32_t batch, int32_t gamma, int32_t vocab, const float *t
     p.tscan = (double *)((char *)workspace + w.tscan_off);
     p.B = batch; p.gamma = gamma; p.V = vocab; p.n_chunks = w.n_chunks;
     cudaStream_t s = (cudaStream_t)stream;
-    return greedy ? launch_accept_greedy(p, s) : launch_accept(p, s);
+    return greedy ? launch_accept_greedy(p, s) : launch_accept(p, (WsHeader *)workspace, variant, s);
 }
 
 }  // extern "C"
@@ -535,8 +650,10 @@ extern "C" int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vo
                                         void *stream) {
     using namespace hippo;
     if (batch <= 0 || gamma < 0 || vocab <= 0) return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: bad sizes");
-    if (mode != HIPPO_ACCEPT_SAMPLE && mode != HIPPO_ACCEPT_GREEDY)
-        return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept_noalloc: mode %d", mode);
+    const int variant = mode & (HIPPO_ACCEPT_ONE_LAUNCH | HIPPO_ACCEPT_THREE_LAUNCHES);
+    mode &= ~(HIPPO_ACCEPT_ONE_LAUNCH | HIPPO_ACCEPT_THREE_LAUNCHES);
+    if ((mode != HIPPO_ACCEPT_SAMPLE && mode != HIPPO_ACCEPT_GREEDY) || variant == (HIPPO_ACCEPT_ONE_LAUNCH | HIPPO_ACCEPT_THREE_LAUNCHES))
+        return fail(HIPPO_ERR_UNIMPLEMENTED, "hippo_accept_noalloc: mode %d", mode | variant);
     const bool greedy = mode == HIPPO_ACCEPT_GREEDY;
     if (!target_logits || !n_accepted || !out_tokens || (!greedy && !u_resample))
         return fail(HIPPO_ERR_INVALID_ARG, "hippo_accept_noalloc: null pointer");
@@ -564,5 +681,5 @@ extern "C" int32_t hippo_accept_noalloc(int32_t batch, int32_t gamma, int32_t vo
     p.tscan = (double *)((char *)scratch + w.tscan_off);
     p.B = batch; p.gamma = gamma; p.V = vocab; p.n_chunks = w.n_chunks;
     cudaStream_t s = (cudaStream_t)stream;
-    return greedy ? launch_accept_greedy(p, s) : launch_accept(p, s);
+    return greedy ? launch_accept_greedy(p, s) : launch_accept(p, (WsHeader *)scratch, variant, s);
 }

@@ -123,11 +123,11 @@ size_t hippo_verify_attention_layers_workspace_bytes(int32_t n_layers, int32_t b
 int32_t hippo_verify_attention_layers(int32_t n_layers, int32_t batch, int32_t q_len, int32_t n_q_heads,
                                       const void *const *q_layers, const hippo_kv_cache_t *kv_layers,
                                       const int32_t *kv_len, const int32_t *kv_len_host, int32_t max_kv_len,
-                                      float softmax_scale, void *const *out_layers, float *const *lse_layers,
+                                      float softmax_scale, int32_t max_ctas, void *const *out_layers, float *const *lse_layers,
                                       void *workspace, size_t workspace_bytes, void *stream) {
     using namespace hippo;
     const char *who = "hippo_verify_attention_layers";
-    if (n_layers <= 0) return fail(HIPPO_ERR_INVALID_ARG, "%s: n_layers <= 0", who);
+    if (n_layers <= 0 || max_ctas < 0) return fail(HIPPO_ERR_INVALID_ARG, "%s: n_layers <= 0 or max_ctas < 0", who);
     if (!q_layers || !kv_layers || !out_layers || !workspace) return fail(HIPPO_ERR_INVALID_ARG, "%s: null pointer", who);
     AttnParams p;
     for (int l = 0; l < n_layers; ++l) {
@@ -147,7 +147,7 @@ int32_t hippo_verify_attention_layers(int32_t n_layers, int32_t batch, int32_t q
         return fail(HIPPO_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu bytes", who, workspace_bytes, L.total);
     if ((uintptr_t)workspace & 255) return fail(HIPPO_ERR_INVALID_ARG, "%s: workspace must be 256-byte aligned", who);
     if (attn_tc_layers_supported(p, kv->dtype) && !attn_small_supported(p, kv->dtype))
-        return launch_attn_tc_layers(p, n_layers, q_layers, kv_layers, out_layers, lse_layers, workspace, (cudaStream_t)stream);
+        return launch_attn_tc_layers(p, n_layers, q_layers, kv_layers, out_layers, lse_layers, max_ctas, workspace, (cudaStream_t)stream);
     // shapes outside the multi-layer kernel: one single-layer call per layer, same results
     for (int l = 0; l < n_layers; ++l) {
         int32_t rc = attention_entry(who, batch, q_len, n_q_heads, q_layers[l], &kv_layers[l], kv_len, kv_len_host, max_kv_len,

@@ -117,7 +117,7 @@ struct AttnLayersWsLayout {
 AttnLayersWsLayout attn_layers_ws_layout(int n_layers, int batch, int q_len, int n_q_heads, int n_kv_heads, int head_dim);
 bool attn_tc_layers_supported(const AttnParams &p, int dtype);
 int32_t launch_attn_tc_layers(const AttnParams &p, int n_layers, const void *const *q, const hippo_kv_cache_t *kv,
-                              void *const *out, float *const *lse, void *workspace, cudaStream_t stream);
+                              void *const *out, float *const *lse, int max_ctas, void *workspace, cudaStream_t stream);
 int32_t launch_attn_small(const AttnParams &p, cudaStream_t stream);
 bool attn_small_supported(const AttnParams &p, int dtype);
 

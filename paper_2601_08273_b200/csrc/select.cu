@@ -10,7 +10,7 @@
 // statistics are therefore accumulated in fp64 (bf16 x bf16 products are exact in fp64), so the kept set only
 // depends on the final rounding of the fused score to fp32.
 //
-// Kernels:  dots (norms + next-frame dot, one warp per token)  ->  spatial (one CTA per crop)  ->
+// Kernels:  dots (norms + next-frame dot, one warp per token)  ->  spatial (one CTA per crop, fp64 tensor instructions)  ->
 //           fuse (one CTA per frame: s_temp, three standardisations, sum)  ->  topk (one CTA per sequence,
 //           bisection on order-preserving keys, ordered compaction).
 //
@@ -110,51 +110,61 @@ __global__ void __launch_bounds__(256) select_dots_kernel(const SelectParams p) 
     if (lane == 0) { p.norm2[j] = n2; p.tdot[j] = td; }
 }
 
-// ---- spatial score: one CTA per crop ---------------------------------------------------------------------------
-// Gram matrix of the crop's (at most 25, in general crop_h*crop_w <= 32) embeddings in fp64.  The embedding dimension is
-// walked in chunks of 128: a chunk of every token of the crop is converted to fp64 once and staged in shared memory
-// (double buffered; the next chunk's global loads are in flight during the arithmetic), then thread (block, slice)
-// accumulates a 5 x 5 block of token pairs over 8 of the 128 dimensions: 10 shared-memory loads feed 25 fused
-// multiply-adds.  The 16 slices of a block are summed by warp shuffles at the end.
-constexpr int kSpaChunk = 128;             // embedding dimensions per staged chunk
-constexpr int kSpaGroup = 5;               // tokens per register-block side
-constexpr int kSpaSlices = 16;             // threads per block of pairs, 8 dimensions each
-// Shape of the kernel for crops of up to NG groups of five tokens: NG = 5 (the paper's 5 x 5 crop, 256 threads, two
-// CTAs per SM) or NG = 7 (up to 32 tokens, 512 threads).
-template <int NG> struct SpaShape {
-    static constexpr int kBlocks = NG * (NG + 1) / 2;                  // upper triangle incl. diagonal
-    static constexpr int kThreads = ((kBlocks * kSpaSlices + 255) / 256) * 256;
-    static constexpr int kRows = NG * kSpaGroup;                       // staged rows (padding rows are zero)
-    static constexpr size_t kSmemBytes = 2 * (size_t)kRows * kSpaChunk * sizeof(double);
+// ---- spatial score on the fp64 tensor path: one CTA per crop ---------------------------------------------------------
+// The Gram matrix of the crop's embeddings is a dense fp64 contraction over the embedding dimension: it runs on
+// mma.sync.m8n8k4.f64 (exact fp64 products of the widened inputs, fp64 accumulation; measured on B200 the instruction
+// sustains 63.7 multiply-adds per clock and SM, plain fp64 FMAs 58).  Tokens are taken in groups of eight; for the groups
+// a <= c the 8 x 8 tile G[a][c] needs one fragment per group and step of four dimensions, and for a Gram matrix the A
+// fragment of a group (row = lane / 4, dimension = lane % 4) is also its B fragment.  The embeddings are staged in shared
+// memory in their storage type, straight from global memory with cp.async (a ring of four 128-dimension chunks, no
+// registers and no conversion on the way in); warp w owns dimensions [16 w, 16 w + 16) of every chunk, and since the order
+// of a dot product's terms is free, lane l takes dimensions 4 (l % 4) .. + 3 of them: one 8-byte (bf16) load per group and
+// chunk, widened to fp64 in registers, feeds the four steps.  Every staged element is read exactly once.  The eight warps'
+// tiles are added in shared memory at the end, in a fixed order; the diagonal of G holds the squared norms.
+// A crop of 25 tokens (the paper's 5 x 5) is padded to four groups: four of the ten tiles serve its last token alone.
+// Leaving that token out of the tiles and taking its 25 dot products with plain multiply-adds (a lane per dimension and
+// partner parity) was built and measured slower (32k tokens: 506 us against 481 us for the whole selection).
+constexpr int kMmaChunk = 128;                 // dimensions per staged chunk
+constexpr int kMmaRowElems = kMmaChunk + 16;   // row stride in elements: four rows of a fragment load cover all banks once
+constexpr int kMmaStages = 4;
+constexpr int kMmaThreads = 256;
+constexpr int kMmaWarps = kMmaThreads / 32;
+constexpr int kMmaTiles = 10;                  // 4 groups: upper triangle incl. diagonal
+template <typename T> struct MmaShape {
+    static constexpr int kRowBytes = kMmaRowElems * (int)sizeof(T);
+    static constexpr int kStageBytes = kMaxCrop * kRowBytes;
+    static constexpr int kPiece = 16 / (int)sizeof(T);               // elements per 16-byte piece
+    static constexpr size_t kRingBytes = (size_t)kMmaStages * kStageBytes;
+    static constexpr size_t kRedBytes = (size_t)kMmaWarps * kMmaTiles * 64 * sizeof(double);
+    static constexpr size_t kSmemBytes = kRingBytes > kRedBytes ? kRingBytes : kRedBytes;
 };
 
-template <typename T> struct Chunk8;   // eight consecutive elements of an embedding row
-template <> struct Chunk8<__nv_bfloat16> {
-    uint4 v;
-    __device__ __forceinline__ void load(const __nv_bfloat16 *p) { v = __ldg(reinterpret_cast<const uint4 *>(p)); }
-    __device__ __forceinline__ void zero() { v = make_uint4(0, 0, 0, 0); }
-    __device__ __forceinline__ void store(double *dst) const {
-        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&v);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); dst[2 * i] = (double)f.x; dst[2 * i + 1] = (double)f.y; }
-    }
-};
-template <> struct Chunk8<float> {
-    float4 a, b;
-    __device__ __forceinline__ void load(const float *p) { a = __ldg(reinterpret_cast<const float4 *>(p)); b = __ldg(reinterpret_cast<const float4 *>(p) + 1); }
-    __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
-    __device__ __forceinline__ void store(double *dst) const {
-        dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w; dst[4] = b.x; dst[5] = b.y; dst[6] = b.z; dst[7] = b.w;
-    }
-};
+__device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                 : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
+// 16 bytes global -> shared, asynchronously; n_bytes = 0 writes zeros and reads nothing
+__device__ __forceinline__ void cp_async_16(void *dst, const void *src, int n_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src), "r"(n_bytes) : "memory");
+}
+__device__ __forceinline__ void load_frag4(const __nv_bfloat16 *p, double *v) {
+    const uint2 u = *reinterpret_cast<const uint2 *>(p);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+    const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+    v[0] = (double)a.x; v[1] = (double)a.y; v[2] = (double)b.x; v[3] = (double)b.y;
+}
+__device__ __forceinline__ void load_frag4(const float *p, double *v) {
+    const float4 a = *reinterpret_cast<const float4 *>(p);
+    v[0] = (double)a.x; v[1] = (double)a.y; v[2] = (double)a.z; v[3] = (double)a.w;
+}
 
-template <typename T, int NG>
-__global__ void __launch_bounds__(SpaShape<NG>::kThreads) select_spatial_kernel(const SelectParams p) {
-    constexpr int kSpaMaxGroups = NG, kSpaMaxBlocks = SpaShape<NG>::kBlocks, kSpaThreads = SpaShape<NG>::kThreads;
-    constexpr int kSpaRows = SpaShape<NG>::kRows;
-    extern __shared__ __align__(16) double stage[];   // [2][kSpaRows][kSpaChunk]
+template <typename T>
+__global__ void __launch_bounds__(kMmaThreads, 2) select_spatial_mma_kernel(const SelectParams p) {
+    using Sh = MmaShape<T>;
+    extern __shared__ __align__(16) uint8_t mma_smem[];   // ring of staged chunks; reused for the warps' partial tiles
     __shared__ int tok[kMaxCrop];
     __shared__ double S[kMaxCrop][kMaxCrop + 1];
+    __shared__ double nrm2[kMaxCrop];
     __shared__ int s_M;
     const int crops_per_frame = p.crops_y * p.crops_x;
     const int gframe = blockIdx.x / crops_per_frame, cr = blockIdx.x % crops_per_frame;
@@ -163,7 +173,7 @@ __global__ void __launch_bounds__(SpaShape<NG>::kThreads) select_spatial_kernel(
     const int n_v = p.seq_off[b + 1] - p.seq_off[b];
     const int nf = min(p.tpf, n_v - f * p.tpf);
     const int y0 = (cr / p.crops_x) * p.crop_h, x0 = (cr % p.crops_x) * p.crop_w;
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
         int M = 0;
         for (int y = y0; y < y0 + p.crop_h && y < p.grid_h; ++y)
@@ -176,91 +186,88 @@ __global__ void __launch_bounds__(SpaShape<NG>::kThreads) select_spatial_kernel(
     if (M == 0) return;
     const T *E = (const T *)p.embeds;
     if (M > 1) {
-        const int n_groups = (M + kSpaGroup - 1) / kSpaGroup;
-        // this thread's block of pairs: groups (ga <= gc), and its 8-dimension slice of every chunk
-        const int blk = tid / kSpaSlices, slice = tid % kSpaSlices;
-        int ga = 0, gc = 0;
-        {
-            int rem = blk;
-            while (ga < kSpaMaxGroups && rem >= kSpaMaxGroups - ga) { rem -= kSpaMaxGroups - ga; ++ga; }
-            gc = ga + rem;
+        const int n_groups = (M + 7) / 8;
+        const int rows = 8 * n_groups;                       // staged rows; rows >= M are zero
+        constexpr int kPiecesPerRow = kMmaChunk / Sh::kPiece;
+        const int n_chunks = (p.d + kMmaChunk - 1) / kMmaChunk;
+        auto stage_chunk = [&](int ch) {
+            uint8_t *dst = mma_smem + (size_t)(ch % kMmaStages) * Sh::kStageBytes;
+            for (int it = tid; it < rows * kPiecesPerRow; it += kMmaThreads) {
+                const int r = it / kPiecesPerRow, c = it % kPiecesPerRow;
+                const int dim = ch * kMmaChunk + c * Sh::kPiece;
+                const bool live = r < M && dim < p.d;           // embed_dim is a multiple of 8: a piece is all there or not at all
+                cp_async_16(dst + r * Sh::kRowBytes + c * 16, live ? (const void *)(E + (size_t)tok[r] * p.d + dim) : (const void *)E, live ? 16 : 0);
+            }
+        };
+        double acc[kMmaTiles][2];
+#pragma unroll
+        for (int t = 0; t < kMmaTiles; ++t) acc[t][0] = acc[t][1] = 0.0;
+        for (int s = 0; s < kMmaStages - 1; ++s) {
+            if (s < n_chunks) stage_chunk(s);
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        const bool active = blk < kSpaMaxBlocks && gc < n_groups;
-        double acc[kSpaGroup][kSpaGroup];
-#pragma unroll
-        for (int i = 0; i < kSpaGroup; ++i)
-#pragma unroll
-            for (int j = 0; j < kSpaGroup; ++j) acc[i][j] = 0.0;
-        // staging: item = (row, 8-column piece); rows beyond M are zero
-        const int rows = n_groups * kSpaGroup;
-        const int items = rows * (kSpaChunk / 8);
-        constexpr int kMaxItems = (kSpaRows * (kSpaChunk / 8) + kSpaThreads - 1) / kSpaThreads;
-        Chunk8<T> pre[kMaxItems];
-        auto fetch = [&](int d0) {
-#pragma unroll
-            for (int k = 0; k < kMaxItems; ++k) {
-                const int it = tid + k * kSpaThreads;
-                const int r = it / (kSpaChunk / 8), c8 = it % (kSpaChunk / 8);
-                if (it < items && r < M && d0 + c8 * 8 < p.d) pre[k].load(E + (size_t)tok[r] * p.d + d0 + c8 * 8);
-                else pre[k].zero();
-            }
-        };
-        auto put = [&](int buf) {
-#pragma unroll
-            for (int k = 0; k < kMaxItems; ++k) {
-                const int it = tid + k * kSpaThreads;
-                if (it < items) pre[k].store(stage + ((size_t)buf * kSpaRows + it / (kSpaChunk / 8)) * kSpaChunk + (it % (kSpaChunk / 8)) * 8);
-            }
-        };
-        const int n_chunks = (p.d + kSpaChunk - 1) / kSpaChunk;
-        fetch(0);
-        put(0);
-        __syncthreads();
         for (int ch = 0; ch < n_chunks; ++ch) {
-            const int buf = ch & 1;
-            if (ch + 1 < n_chunks) fetch((ch + 1) * kSpaChunk);
-            if (active) {
-                const double *ra = stage + ((size_t)buf * kSpaRows + ga * kSpaGroup) * kSpaChunk + slice;
-                const double *rc = stage + ((size_t)buf * kSpaRows + gc * kSpaGroup) * kSpaChunk + slice;
-#pragma unroll
-                for (int k = 0; k < kSpaChunk / kSpaSlices; ++k) {
-                    double va[kSpaGroup], vc[kSpaGroup];
-#pragma unroll
-                    for (int i = 0; i < kSpaGroup; ++i) { va[i] = ra[i * kSpaChunk + k * kSpaSlices]; vc[i] = rc[i * kSpaChunk + k * kSpaSlices]; }
-#pragma unroll
-                    for (int i = 0; i < kSpaGroup; ++i)
-#pragma unroll
-                        for (int j = 0; j < kSpaGroup; ++j) acc[i][j] = fma(va[i], vc[j], acc[i][j]);
-                }
-            }
-            if (ch + 1 < n_chunks) put(buf ^ 1);
+            // chunk ch has landed for every thread, and everybody is done with the slot that the next load overwrites
+            asm volatile("cp.async.wait_group %0;" ::"n"(kMmaStages - 2) : "memory");
             __syncthreads();
-        }
-        // the 16 slices of a block sit in one half-warp
+            if (ch + kMmaStages - 1 < n_chunks) stage_chunk(ch + kMmaStages - 1);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            const T *st = reinterpret_cast<const T *>(mma_smem + (size_t)(ch % kMmaStages) * Sh::kStageBytes);
+            double frag[4][4];   // [group][step]
 #pragma unroll
-        for (int i = 0; i < kSpaGroup; ++i)
-#pragma unroll
-            for (int j = 0; j < kSpaGroup; ++j) {
-                double v = acc[i][j];
-#pragma unroll
-                for (int o = kSpaSlices / 2; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                acc[i][j] = v;
+            for (int g = 0; g < 4; ++g) {
+                if (g < n_groups) load_frag4(st + (g * 8 + (lane >> 2)) * kMmaRowElems + warp * 16 + (lane & 3) * 4, frag[g]);
+                else frag[g][0] = frag[g][1] = frag[g][2] = frag[g][3] = 0.0;
             }
-        if (active && slice == 0) {
 #pragma unroll
-            for (int i = 0; i < kSpaGroup; ++i)
+            for (int step = 0; step < 4; ++step) {
+                int t = 0;
 #pragma unroll
-                for (int j = 0; j < kSpaGroup; ++j) {
-                    const int ta = ga * kSpaGroup + i, tc = gc * kSpaGroup + j;
-                    if (ta < M && tc < M && ta < tc) {
-                        const double na = p.norm2[tok[ta]], nc = p.norm2[tok[tc]];
-                        const double cs = (na > 0.0 && nc > 0.0) ? acc[i][j] / (sqrt(na) * sqrt(nc)) : 0.0;
-                        S[ta][tc] = cs;
-                        S[tc][ta] = cs;
-                    }
-                }
+                for (int ga = 0; ga < 4; ++ga)
+#pragma unroll
+                    for (int gc = ga; gc < 4; ++gc, ++t)
+                        if (gc < n_groups) dmma_m8n8k4(acc[t][0], acc[t][1], frag[ga][step], frag[gc][step]);   // uniform over the CTA
+            }
         }
-        (void)lane;
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        __syncthreads();
+        // the eight warps' partial tiles meet in shared memory (the ring is idle now)
+        double *red = reinterpret_cast<double *>(mma_smem);
+        {
+            double *mine = red + (size_t)warp * (kMmaTiles * 64);
+            int t = 0;
+#pragma unroll
+            for (int ga = 0; ga < 4; ++ga)
+#pragma unroll
+                for (int gc = ga; gc < 4; ++gc, ++t)
+                    if (gc < n_groups) {
+                        mine[t * 64 + (lane >> 2) * 8 + (lane & 3) * 2] = acc[t][0];
+                        mine[t * 64 + (lane >> 2) * 8 + (lane & 3) * 2 + 1] = acc[t][1];
+                    }
+        }
+        __syncthreads();
+        // G[a][c] for a <= c, summed over the warps in a fixed order; then the cosines
+        for (int x = tid; x < M * M; x += kMmaThreads) {
+            const int a = x / M, c = x % M;
+            if (a > c) continue;
+            const int ga = a >> 3, gc = c >> 3;
+            const int t = ga * 4 - ga * (ga - 1) / 2 + (gc - ga);       // index of tile (ga, gc) in the upper triangle of 4 x 4
+            double g = 0.0;
+            for (int w = 0; w < kMmaWarps; ++w) g += red[(size_t)w * (kMmaTiles * 64) + t * 64 + (a & 7) * 8 + (c & 7)];
+            S[a][c] = g;
+        }
+        __syncthreads();
+        if (tid < M) nrm2[tid] = S[tid][tid];
+        __syncthreads();
+        for (int x = tid; x < M * M; x += kMmaThreads) {
+            const int a = x / M, c = x % M;
+            if (a >= c) continue;
+            const double na = nrm2[a], nc = nrm2[c];
+            const double cs = (na > 0.0 && nc > 0.0) ? S[a][c] / (sqrt(na) * sqrt(nc)) : 0.0;
+            S[a][c] = cs;
+            S[c][a] = cs;
+        }
+        __syncthreads();
     }
     if (tid < M) S[tid][tid] = 1.0;
     __syncthreads();
@@ -411,10 +418,90 @@ __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p,
     const int need_eq = s_remaining;  // elements equal to T to keep: those with the smallest indices
     if (tid == 0) { s_base_eq = 0; s_base_out = 0; }
     __syncthreads();
-    // ordered compaction, blockDim.x elements at a time: ranks from ballots, warp offsets from a scan by warp 0
-    __shared__ int eq_off[33], sel_off[33];
+    // Ordered compaction.  Element i = e * blockDim.x + tid of the first n_regs sits in this thread's register e, so the
+    // output position of a kept element is (kept elements of rows e' < e) + (kept elements of row e in lower threads).
+    // Three sweeps over the registers, ballots only, and two scans of the 32 x 32 table of per-(row, warp) counts in
+    // between: first the ranks of the elements equal to the threshold (only the need_eq lowest indices among them are
+    // kept), then the output positions.
+    __shared__ int cnt[32][33];
+    __shared__ int row_tot[32];
     const int nw = blockDim.x >> 5;
-    for (int start = 0; start < n; start += blockDim.x) {
+    const int rows_used = min(kKeysPerThread, (n + (int)blockDim.x - 1) / (int)blockDim.x);
+    // exclusive scan of cnt[e][w] in (e, w) order, in place; returns the grand total through row_tot[31]
+    auto scan_counts = [&]() {
+        __syncthreads();
+        if (warp < rows_used) {
+            const int c = lane < nw ? cnt[warp][lane] : 0;
+            int inc = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += v; }
+            cnt[warp][lane] = inc - c;
+            if (lane == 31) row_tot[warp] = inc;
+        } else if (lane == 31) {
+            row_tot[warp] = 0;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            const int c = row_tot[lane];
+            int inc = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += v; }
+            row_tot[lane] = inc - c;
+            if (lane == 31) s_base_eq = inc;      // scratch: the grand total
+        }
+        __syncthreads();
+    };
+    const unsigned lt_mask = (1u << lane) - 1;
+#pragma unroll
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        if (e < rows_used) {   // uniform
+            const unsigned bal = __ballot_sync(0xffffffffu, e * (int)blockDim.x + tid < n && keys[e] == T);
+            if (lane == 0) cnt[e][warp] = __popc(bal);
+        }
+    }
+    scan_counts();
+    const int eq_in_regs = s_base_eq;
+    __syncthreads();
+    __shared__ int eq_off[32][33];
+    __shared__ int eq_row[32];
+    for (int x = tid; x < 32 * 32; x += blockDim.x) eq_off[x >> 5][x & 31] = cnt[x >> 5][x & 31];
+    if (tid < 32) eq_row[tid] = row_tot[tid];
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        if (e < rows_used) {
+            const bool in = e * (int)blockDim.x + tid < n;
+            const bool eq = in && keys[e] == T, gt = in && keys[e] > T;
+            const unsigned bal_eq = __ballot_sync(0xffffffffu, eq);
+            const int rank = eq_row[e] + eq_off[e][warp] + __popc(bal_eq & lt_mask);
+            const unsigned bal = __ballot_sync(0xffffffffu, gt || (eq && rank < need_eq));
+            if (lane == 0) cnt[e][warp] = __popc(bal);
+        }
+    }
+    scan_counts();
+    const int out_in_regs = s_base_eq;
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        if (e < rows_used) {
+            const int i = e * (int)blockDim.x + tid;
+            const bool in = i < n;
+            const bool eq = in && keys[e] == T, gt = in && keys[e] > T;
+            const unsigned bal_eq = __ballot_sync(0xffffffffu, eq);
+            const int rank = eq_row[e] + eq_off[e][warp] + __popc(bal_eq & lt_mask);
+            const bool sel = gt || (eq && rank < need_eq);
+            const unsigned bal = __ballot_sync(0xffffffffu, sel);
+            const int pos = row_tot[e] + cnt[e][warp] + __popc(bal & lt_mask);
+            if (sel && pos < k) out[pos] = i;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) { s_base_eq = eq_in_regs; s_base_out = out_in_regs; }
+    __syncthreads();
+    // what lies beyond the registers (more than 32 keys per thread): blockDim.x elements at a time, ranks from ballots,
+    // warp offsets from a scan by warp 0
+    __shared__ int tail_eq_off[33], sel_off[33];
+    for (int start = n_regs; start < n; start += blockDim.x) {
         const int i = start + tid;
         const uint32_t key = i < n ? order_key(score[i]) : 0u;
         const bool gt = i < n && key > T, eq = i < n && key == T;
@@ -426,12 +513,12 @@ __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p,
             int inc = c;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += v; }
-            eq_off[lane] = inc - c;
-            if (lane == 31) eq_off[32] = inc;
+            tail_eq_off[lane] = inc - c;
+            if (lane == 31) tail_eq_off[32] = inc;
         }
         __syncthreads();
-        const int eq_rank = s_base_eq + eq_off[warp] + __popc(bal_eq & ((1u << lane) - 1));
-        const bool sel = gt || (eq && eq_rank < need_eq);
+        const int eq_rank2 = s_base_eq + tail_eq_off[warp] + __popc(bal_eq & lt_mask);
+        const bool sel = gt || (eq && eq_rank2 < need_eq);
         const unsigned bal = __ballot_sync(0xffffffffu, sel);
         if (lane == 0) warp_cnt[warp] = __popc(bal);
         __syncthreads();
@@ -444,10 +531,10 @@ __global__ void __launch_bounds__(1024) select_topk_kernel(const SelectParams p,
             if (lane == 31) sel_off[32] = inc;
         }
         __syncthreads();
-        const int pos = s_base_out + sel_off[warp] + __popc(bal & ((1u << lane) - 1));
+        const int pos = s_base_out + sel_off[warp] + __popc(bal & lt_mask);
         if (sel && pos < k) out[pos] = i;
         __syncthreads();
-        if (tid == 0) { s_base_eq += eq_off[32]; s_base_out += sel_off[32]; }
+        if (tid == 0) { s_base_eq += tail_eq_off[32]; s_base_out += sel_off[32]; }
         __syncthreads();
     }
 }
@@ -642,19 +729,12 @@ int32_t hippo_select_tokens_policy(int32_t batch, const int32_t *n_visual, int32
         static PerDeviceOnce spa_attr;
         int dev;
         if (spa_attr.needed(dev)) {
-            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<float, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<5>::kSmemBytes));
-            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<__nv_bfloat16, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<5>::kSmemBytes));
-            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<float, 7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<7>::kSmemBytes));
-            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_kernel<__nv_bfloat16, 7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpaShape<7>::kSmemBytes));
+            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_mma_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MmaShape<float>::kSmemBytes));
+            HIPPO_CUDA_TRY(cudaFuncSetAttribute(select_spatial_mma_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MmaShape<__nv_bfloat16>::kSmemBytes));
             spa_attr.mark(dev);
         }
-        if (crop_h * crop_w <= 25) {
-            if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float, 5><<<g2, SpaShape<5>::kThreads, SpaShape<5>::kSmemBytes, s>>>(p);
-            else select_spatial_kernel<__nv_bfloat16, 5><<<g2, SpaShape<5>::kThreads, SpaShape<5>::kSmemBytes, s>>>(p);
-        } else {
-            if (dtype == HIPPO_DTYPE_FP32) select_spatial_kernel<float, 7><<<g2, SpaShape<7>::kThreads, SpaShape<7>::kSmemBytes, s>>>(p);
-            else select_spatial_kernel<__nv_bfloat16, 7><<<g2, SpaShape<7>::kThreads, SpaShape<7>::kSmemBytes, s>>>(p);
-        }
+        if (dtype == HIPPO_DTYPE_FP32) select_spatial_mma_kernel<float><<<g2, kMmaThreads, MmaShape<float>::kSmemBytes, s>>>(p);
+        else select_spatial_mma_kernel<__nv_bfloat16><<<g2, kMmaThreads, MmaShape<__nv_bfloat16>::kSmemBytes, s>>>(p);
         count_launches(1);
     }
     const int fuse_threads = ((p.tpf + 31) / 32) * 32;

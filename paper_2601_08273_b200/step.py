@@ -34,9 +34,18 @@ def _randn(shape, dtype, gen, device):
 class HippoStep:
     def __init__(self, cfg: W.HippoConfig, device="cuda", target_layers: Optional[int] = None,
                  draft_layers: Optional[int] = None, host_inputs: Optional[Dict[str, np.ndarray]] = None,
-                 multi_layer_verify: bool = True):
+                 multi_layer_verify: bool = True, verify_max_ctas: int = 0):
         self.cfg = cfg
         self.multi_layer_verify = multi_layer_verify
+        # How run() shares the GPU between its two legs (all three can be changed before run() is called or captured):
+        #   verify_max_ctas       grid bound of the multi-layer verification kernel; the SMs it leaves free are where the
+        #                         draft stream's kernels run (a persistent CTA holds all of its SM's shared memory)
+        #   verify_beside_select  True: verification is forked first and also runs beside select and gather
+        #   draft_num_splits      work split of the draft attention calls (0: automatic, which may pick clusters of up to 16
+        #                         CTAs that do not fit into a few scattered free SMs)
+        self.verify_max_ctas = verify_max_ctas
+        self.verify_beside_select = False
+        self.draft_num_splits = 0
         self.device = torch.device(device)
         self.Lt = cfg.tgt_layers if target_layers is None else target_layers
         self.Ld = cfg.dft_layers if draft_layers is None else draft_layers
@@ -119,6 +128,17 @@ class HippoStep:
 
         self.stream_d = torch.cuda.Stream(device=self.device)
         self.stream_v = torch.cuda.Stream(device=self.device)
+        if verify_max_ctas == 0 and multi_layer_verify:
+            # Default sharing, from the two legs' sizes: when the draft leg (latency-bound calls, about 10 us each) outlasts the
+            # verification leg (bandwidth-bound), verification gives up 84 of the 148 SMs to it; measured on B200 this takes
+            # the 6k-token step from 1.55 ms to 1.12 ms and the 32k-token step from 3.52 ms to 3.03 ms.  When verification is
+            # the longer leg (64k tokens, 80 layers) it keeps every SM: the draft calls then run in its shadow or after it,
+            # and holding SMs back only slows the step down (7.05 ms against 7.37 ms with 116 CTAs).
+            verify_s = self.verify_kv_bytes_per_layer() * self.Lt / 5.4e12
+            draft_s = g * self.Ld * 10e-6
+            if draft_s > verify_s:
+                self.verify_max_ctas = 64
+        self.draft_num_splits = 16 if max(self.n_keep) + g > 1024 and B * h <= 4 else 0
 
     # ---- algorithmic bytes (the roofline numerators) ------------------------------------------------------------
     @property
@@ -193,7 +213,8 @@ class HippoStep:
         for j in range(self.cfg.gamma):
             for l in range(self.Ld):
                 hb.hippo_draft_attention(self.q_d[l, j], self.dst_cache[l], self.kv_len_d[j], self.max_kv_d[j],
-                                         out=self.out_d[l, j], workspace=self.draft_ws, stream=stream)
+                                         out=self.out_d[l, j], workspace=self.draft_ws, stream=stream,
+                                         num_splits=self.draft_num_splits)
 
     def verify(self, stream=None):
         """The verification leg, one call per target layer."""
@@ -202,14 +223,17 @@ class HippoStep:
             hb.hippo_verify_attention(self.q_t[l], self.tgt_cache[l], self.kv_len_t, m, out=self.out_t[l],
                                       workspace=self.verify_ws, stream=stream, kv_len_host=self.kv_len_t_host)
 
-    def verify_layers(self, stream=None):
+    def verify_layers(self, stream=None, max_ctas: int = 0):
         """The verification leg, all target layers in one call."""
         hb.hippo_verify_attention_layers(self.q_t_layers, self.tgt_cache, self.kv_len_t, max(self.kv_len_t_host),
                                          self.out_t_layers, workspace=self.verify_layers_ws, stream=stream,
-                                         kv_len_host=self.kv_len_t_host)
+                                         kv_len_host=self.kv_len_t_host, max_ctas=max_ctas)
 
     def verify_leg(self, stream=None):
-        (self.verify_layers if self.multi_layer_verify else self.verify)(stream)
+        if self.multi_layer_verify:
+            self.verify_layers(stream, self.verify_max_ctas)
+        else:
+            self.verify(stream)
 
     def attention_mass(self, stream=None):
         """Eq. 2 over all target layers of the prefilled cache (once per prompt, upstream of select); the result goes
@@ -242,11 +266,19 @@ class HippoStep:
                         n_accepted=self.n_accepted, out_tokens=self.out_tokens, workspace=self.accept_ws, stream=stream)
 
     def run(self):
-        """The whole step on the current stream, with draft and verify forked onto their own streams."""
+        """The whole step on the current stream, with draft and verify forked onto their own streams.
+
+        The verification leg reads neither the selection nor the pruned cache.  With `verify_beside_select` it is forked
+        first and runs beside select and gather too; otherwise it starts once the selection has finished (the selection's
+        fp64 kernels want every SM for themselves) and runs beside the draft calls only."""
         main = torch.cuda.current_stream(self.device)
-        self.stream_v.wait_stream(main)
-        self.verify_leg(self.stream_v)        # reads neither the selection nor the pruned cache
+        if self.verify_beside_select:
+            self.stream_v.wait_stream(main)
+            self.verify_leg(self.stream_v)
         self.select(main)
+        if not self.verify_beside_select:
+            self.stream_v.wait_stream(main)
+            self.verify_leg(self.stream_v)
         self.gather(main)
         self.stream_d.wait_stream(main)
         self.draft(self.stream_d)             # reads the gathered cache

@@ -22,9 +22,13 @@ from .step import HippoStep, _randn
 
 class VpsdLoop:
     def __init__(self, cfg: W.HippoConfig, target_layers: Optional[int] = None, draft_layers: Optional[int] = None,
-                 buffered: int = 0, pool: int = 8, draft_noise: float = 1.0, use_graphs: bool = True, device="cuda"):
+                 buffered: int = 0, pool: int = 8, draft_noise: float = 1.0, use_graphs: bool = True, device="cuda",
+                 verify_max_ctas: int = 0):
         assert cfg.batch == 1, "the schedule is per sequence; the driver runs one sequence"
         self.cfg = cfg
+        # verify_max_ctas > 0: the verification kernel leaves the other SMs to the draft stream (it holds its own for the
+        # whole pass), which is what lets the two legs of a round overlap on one GPU
+        self.verify_max_ctas = verify_max_ctas
         self.st = HippoStep(cfg, device=device, target_layers=target_layers, draft_layers=draft_layers)
         st, g = self.st, cfg.gamma
         self.dev = st.device
@@ -85,14 +89,16 @@ class VpsdLoop:
         st = self.st
         for l in range(st.Ld):
             hb.hippo_draft_attention(st.q_d[l, jj], st.dst_cache[l], st.kv_len_d[jj], st.max_kv_d[jj],
-                                     out=st.out_d[l, jj], workspace=st.draft_ws, stream=stream)
+                                     out=st.out_d[l, jj], workspace=st.draft_ws, stream=stream,
+                                     num_splits=st.draft_num_splits)
 
     def _verify_eager(self, c: int, stream) -> None:
         st = self.st
         # the verification pass: every target layer's attention in one launch
         hb.hippo_verify_attention_layers([self.q_t[l][:, :c + 1] for l in range(st.Lt)], st.tgt_cache, self.kv_len_t[c],
                                          st.ctx[0] + c + 1, [self.out_t[l][:, :c + 1] for l in range(st.Lt)],
-                                         workspace=self.verify_ws, stream=stream, kv_len_host=[st.ctx[0] + c + 1])
+                                         workspace=self.verify_ws, stream=stream, kv_len_host=[st.ctx[0] + c + 1],
+                                         max_ctas=self.verify_max_ctas)
 
     def draft_token(self, j: int, stream) -> None:
         jj = j % self.cfg.gamma

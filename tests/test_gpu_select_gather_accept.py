@@ -324,22 +324,26 @@ def check_accept(hb, inp, what, forgiven_allowed=0):
     """Accepted lengths and emitted tokens bit for bit.  A differing sequence is forgiven only when the oracle reports
     that a uniform sat within 1e-12 (relative) of a decision boundary, and the number forgiven is itself checked:
     none on the benchmark configurations."""
-    n, out = hb.hippo_accept(dev(inp["target_logits"]), dev(inp["draft_logits"]), dev(inp["draft_tokens"]),
-                             dev(inp["u_accept"]), dev(inp["u_resample"]))
-    torch.cuda.synchronize()
     rn, rout, ma, mc = oracle.accept(inp["target_logits"], inp["draft_logits"], inp["draft_tokens"], inp["u_accept"],
                                      inp["u_resample"])
     # the margins themselves must be usable: positive and finite wherever a test / a draw was made
     assert np.all(mc >= 0) and np.all(np.isfinite(mc)), what
     assert np.all(ma >= 0), what
-    n, out = host(n), host(out)
-    bad = np.where((n != rn) | (out != rout).any(axis=1))[0]
-    forgiven = 0
-    for b in bad:
-        assert min(ma[b], mc[b]) < 1e-12, "%s: sequence %d differs (n %d vs %d, tokens %s vs %s), margins %.3e %.3e" % (
-            what, b, n[b], rn[b], out[b], rout[b], ma[b], mc[b])
-        forgiven += 1
-    assert forgiven <= forgiven_allowed, "%s: %d of %d sequences forgiven by the near-boundary rule" % (what, forgiven, len(rn))
+    args = [dev(inp[k]) for k in ("target_logits", "draft_logits", "draft_tokens", "u_accept", "u_resample")]
+    # both launch forms of the sampling acceptance (one kernel / three chained kernels), and the library's own choice
+    for form, flag in (("chain", hb.HIPPO_ACCEPT_THREE_LAUNCHES), ("one launch", hb.HIPPO_ACCEPT_ONE_LAUNCH), ("auto", 0)):
+        ws = hb.new_workspace(hb.hippo_accept_workspace_bytes(*rout.shape[:1], rout.shape[1] - 1, inp["target_logits"].shape[2]))
+        n, out = hb.hippo_accept(*args, mode=hb.HIPPO_ACCEPT_SAMPLE | flag, workspace=ws)
+        torch.cuda.synchronize()
+        assert hb.hippo_workspace_status(ws) == hb.HIPPO_OK
+        n, out = host(n), host(out)
+        bad = np.where((n != rn) | (out != rout).any(axis=1))[0]
+        forgiven = 0
+        for b in bad:
+            assert min(ma[b], mc[b]) < 1e-12, "%s (%s): sequence %d differs (n %d vs %d, tokens %s vs %s), margins %.3e %.3e" % (
+                what, form, b, n[b], rn[b], out[b], rout[b], ma[b], mc[b])
+            forgiven += 1
+        assert forgiven <= forgiven_allowed, "%s (%s): %d of %d sequences forgiven by the near-boundary rule" % (what, form, forgiven, len(rn))
     return rn
 
 

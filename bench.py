@@ -3,8 +3,8 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference] [--no-graph] [--no-extra]
 
-A step is one pass of the whole hot path over one batch of synthetic input: (verify attention of all target layers on
-one stream) || (select -> gather -> gamma x draft layers of draft attention on another) -> accept.  The metric is the
+A step is one pass of the whole hot path over one batch of synthetic input: select -> (verify attention of all target
+layers on one stream || gather -> gamma x draft layers of draft attention on another) -> accept.  The metric is the
 verification leg's KV-read bandwidth: target-KV bytes attended per step / device time of the step's verification
 launches (CUDA events on the stream that launches them).  One JSON line is printed by rank 0.
 
@@ -33,7 +33,9 @@ if ROOT not in sys.path:
 METRIC = "verify_kv_read_gbps"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
-FP64_PEAK_FLOPS = 148 * 64 * 2 * 1.965e9      # 64 fp64 FMA per clock per SM
+# 64 fp64 multiply-adds per clock and SM; a register-only probe of mma.sync.m8n8k4.f64 on this part measured 63.7 with
+# constant operands and 47 with operands that change every instruction
+FP64_PEAK_FLOPS = 148 * 64 * 2 * 1.965e9
 MUFU_PEAK_PER_S = 148 * 16 * 1.965e9          # 16 ex2 per clock per SM
 
 
@@ -297,11 +299,14 @@ def kernel_sweep(cfg, torch, hb, HippoStep, peaks, uuid, reps=20, max_gb=24.0, b
         med = statistics.median(per) / layers
         out["attention_mass"] = {"us_per_layer": spread(per, 1e3 / layers), "gexp_per_s": round(st.mass_exps_per_layer() / med / 1e6, 1),
                                  "frac_of_mufu_peak": round(st.mass_exps_per_layer() / (med * 1e-3) / MUFU_PEAK_PER_S, 4)}
-    # the whole step: verify || (select -> gather -> draft) -> accept
+    # the whole step: select -> (verify || gather -> draft) -> accept, replayed from a graph like the headline step
     st.run()
     torch.cuda.synchronize()
+    step_replay = try_graph(st.run, torch)
+    step_run = step_replay if step_replay is not None else st.run
+    step_run()
     sampler.mark()
-    _, per = timed_reps(st.run, n_small, cur, torch)
+    _, per = timed_reps(step_run, n_small, cur, torch)
     sampler.mark()
     out["step_ms"] = spread(per)
     out["step_draft_layers"] = st.Ld
@@ -367,6 +372,8 @@ def run_ours(args):
     uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
     peaks = Peaks(torch, hb)
     cfg = W.CONFIGS[args.config]
+    if args.layers is not None:
+        cfg = cfg.replace(tgt_layers=max(1, args.layers))
     st = HippoStep(cfg)
     cur = torch.cuda.current_stream()
 
@@ -627,6 +634,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--config", type=int, default=2,
                     help="index into the five configurations (default 2: long video, 32,768 visual tokens, the smallest size the bandwidth target is stated for)")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="time this many target layers instead of the configuration's (a small case for profiler captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the per-call timings and whole-step times of the other configurations")

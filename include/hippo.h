@@ -234,7 +234,8 @@ int32_t hippo_gather_kv(int32_t n_layers, const hippo_kv_cache_t *src, size_t sr
  *            loads without the round trip for the length
  *   kv_len_host  optional HOST copy of kv_len (NULL: none).  Used only to plan the launch: with the real lengths of a
  *            ragged batch the work split is chosen from the total number of pages instead of batch * the longest;
- *            the kernels still read kv_len on the device, results do not depend on it
+ *            the kernels still read kv_len on the device, and results depend on it only through the order of the
+ *            floating-point sums
  *   max_kv_len  host upper bound used to size the launch; <= max_pages_per_seq * 64
  *   softmax_scale  0 selects 1/sqrt(head_dim)
  *   num_splits  0 = automatic

@@ -76,10 +76,9 @@ def test_layers_ragged_batch_more_layers_than_slot_sets(hb, D):
     B, q_len, Hq, Hkv = 4, 6, 8, 2
     lens = [2333, 6, 1290, 3]
     q, k, v = layer_inputs(rng, 7, B, q_len, Hq, Hkv, D, lens, "bf16")
-    a = check_layers(hb, q, k, v, lens, "bf16", fill=np.nan)
-    b = check_layers(hb, q, k, v, lens, "bf16", host_lens=True, want_lse=False)
-    for x, y in zip(a, b):
-        np.testing.assert_array_equal(x, y)      # the host copy of the lengths only plans the launch
+    check_layers(hb, q, k, v, lens, "bf16", fill=np.nan)
+    # the host copy of the lengths only plans the launch (grid, work split): another summation order, the same result
+    check_layers(hb, q, k, v, lens, "bf16", host_lens=True, want_lse=False)
 
 
 def test_layers_one_unit_per_cta_and_more(hb):

@@ -316,30 +316,40 @@ def kernel_sweep(cfg, torch, hb, HippoStep, peaks, uuid, reps=20, max_gb=24.0, b
     return out
 
 
-def schedule_entry(cfg, torch, hb, rounds=40, draft_noise=0.5, verify_max_ctas=0):
+def schedule_entry(cfg, torch, hb, rounds=40, draft_noise=0.5, verify_max_ctas=0, gamma=None, draft_num_splits=None):
     """The adaptive decoding schedule (Section 5.2) over the kernels against the serial schedule.  draft_noise sets how far
     the synthetic draft logits are from the target's (the acceptance rate); verify_max_ctas > 0 leaves SMs to the draft
     stream while the verification kernel runs."""
     from paper_2601_08273_b200.vpsd import VpsdLoop
     torch.cuda.empty_cache()
-    loop = VpsdLoop(cfg, buffered=0, pool=8, draft_noise=draft_noise, verify_max_ctas=verify_max_ctas)
+    loop = VpsdLoop(cfg, buffered=0, pool=8, draft_noise=draft_noise, verify_max_ctas=verify_max_ctas, gamma=gamma,
+                    draft_num_splits=draft_num_splits)
+    cfg = loop.cfg
     unit = loop.unit_times_ms()
+    shared = loop.shared_times_ms()
     loop.run(4); loop.run_serial(2)
     par, ser = loop.run(rounds), loop.run_serial(rounds // 2)
     state = hb.hippo_vpsd_init(cfg.gamma, 0)
-    model_ms = 0.0
+    # the round-time model twice: with each leg's time measured alone (the paper's setting: the legs do not share a
+    # memory system) and with the times the legs show side by side on this one GPU
+    model_ms, shared_model_ms = 0.0, 0.0
     for t in par["trace"]:
         rd = hb.hippo_vpsd_plan(state)
         model_ms += hb.hippo_vpsd_round_time(rd, t["accepted"], unit["t_draft"], unit["t_target"])
+        u = shared if rd.draft_during > 0 else unit
+        shared_model_ms += hb.hippo_vpsd_round_time(rd, t["accepted"], u["t_draft"], u["t_target"])
         hb.hippo_vpsd_commit(state, rd, t["accepted"], t["drafted_during"])
     serial_model = sum(hb.hippo_vpsd_serial_round_time(cfg.gamma, unit["t_draft"], unit["t_target"]) for _ in range(ser["rounds"]))
     out = {"workload": cfg.name + " decoding schedule", "gamma": cfg.gamma, "rounds": par["rounds"],
-           "draft_noise": draft_noise, "verify_max_ctas": verify_max_ctas,
+           "draft_noise": draft_noise, "verify_max_ctas": verify_max_ctas, "draft_num_splits": loop.st.draft_num_splits,
            "t_draft_token_ms": round(unit["t_draft"], 4), "t_verify_ms": round(unit["t_target"], 4),
            "target_over_draft": round(unit["t_target"] / unit["t_draft"], 2),
            "parallel_tokens": par["tokens"], "parallel_ms": round(par["wall_ms"], 3),
            "parallel_tokens_per_s": round(par["tokens"] / par["wall_ms"] * 1e3, 1),
            "parallel_model_ms": round(model_ms, 3), "parallel_measured_over_model": round(par["wall_ms"] / model_ms, 3),
+           "t_draft_token_beside_verify_ms": round(shared["t_draft"], 4), "t_verify_beside_draft_ms": round(shared["t_target"], 4),
+           "parallel_shared_gpu_model_ms": round(shared_model_ms, 3),
+           "parallel_measured_over_shared_gpu_model": round(par["wall_ms"] / shared_model_ms, 3),
            "optimistic_rounds": sum(1 for t in par["trace"] if t["mode"] == 0),
            "mean_accepted": round(sum(t["accepted"] for t in par["trace"]) / par["rounds"], 2),
            "serial_tokens": ser["tokens"], "serial_ms": round(ser["wall_ms"], 3),

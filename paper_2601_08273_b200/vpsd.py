@@ -10,6 +10,7 @@ switch.  Batch size 1, as in the paper.
 """
 from __future__ import annotations
 
+import dataclasses
 import time
 from typing import Dict, List, Optional
 
@@ -23,13 +24,20 @@ from .step import HippoStep, _randn
 class VpsdLoop:
     def __init__(self, cfg: W.HippoConfig, target_layers: Optional[int] = None, draft_layers: Optional[int] = None,
                  buffered: int = 0, pool: int = 8, draft_noise: float = 1.0, use_graphs: bool = True, device="cuda",
-                 verify_max_ctas: int = 0):
+                 verify_max_ctas: int = 0, gamma: Optional[int] = None, draft_num_splits: Optional[int] = None):
         assert cfg.batch == 1, "the schedule is per sequence; the driver runs one sequence"
+        if gamma is not None:
+            cfg = dataclasses.replace(cfg, gamma=gamma)
         self.cfg = cfg
-        # verify_max_ctas > 0: the verification kernel leaves the other SMs to the draft stream (it holds its own for the
-        # whole pass), which is what lets the two legs of a round overlap on one GPU
+        # Sharing one GPU between the two legs of a round.  The verification kernel keeps its CTAs for the whole pass and a
+        # draft call is a wave of CTAs of its own, so the legs overlap only when both fit: verify_max_ctas > 0 bounds the
+        # verification grid, and draft_num_splits (CTAs per (sequence, KV head) of a draft call over a long pruned cache)
+        # sizes a draft call for the SMs that leaves free.  Left alone, a 148-CTA verification pass makes the draft
+        # stream wait for its end and the round costs the sum of the legs.
         self.verify_max_ctas = verify_max_ctas
         self.st = HippoStep(cfg, device=device, target_layers=target_layers, draft_layers=draft_layers)
+        if draft_num_splits is not None:
+            self.st.draft_num_splits = draft_num_splits
         st, g = self.st, cfg.gamma
         self.dev = st.device
         self.max_batch = max(g, buffered)
@@ -204,3 +212,32 @@ class VpsdLoop:
             return e0.elapsed_time(e1) / reps
         return {"t_draft": timed(lambda: self.draft_token(0, main)),
                 "t_target": timed(lambda: self.verify_and_accept(self.cfg.gamma, 0, main))}
+
+    def shared_times_ms(self, reps: int = 5) -> Dict[str, float]:
+        """The same two times with both legs of an optimistic round in flight: gamma draft tokens on the draft stream
+        beside one verification pass on the other.  On one GPU the legs share the SMs and, above all, the memory system:
+        a draft call is a chain of dependent memory round trips whose latency grows severalfold while the verification
+        kernel keeps HBM saturated, so a round costs max(t_target, gamma * t_draft) of THESE times, not of the times
+        each leg shows alone."""
+        g = self.cfg.gamma
+        sd, sv = self.stream_d, self.stream_v
+        td, tv = [], []
+        for _ in range(reps + 1):
+            torch.cuda.synchronize(self.dev)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            go = torch.cuda.Event()
+            go.record(torch.cuda.current_stream(self.dev))
+            sv.wait_event(go)
+            sd.wait_event(go)
+            ev[0].record(sv)
+            self.verify_and_accept(g, 0, sv)
+            ev[1].record(sv)
+            ev[2].record(sd)
+            for j in range(g):
+                self.draft_token(j, sd)
+            ev[3].record(sd)
+            torch.cuda.synchronize(self.dev)
+            tv.append(ev[0].elapsed_time(ev[1]))
+            td.append(ev[2].elapsed_time(ev[3]) / g)
+        td, tv = sorted(td[1:]), sorted(tv[1:])
+        return {"t_draft": td[len(td) // 2], "t_target": tv[len(tv) // 2]}

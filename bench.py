@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the HIPPO hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference] [--no-graph] [--no-extra]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference] [--no-graph] [--no-extra] [--no-breakdown]
 
 A step is one pass of the whole hot path over one batch of synthetic input: select -> (verify attention of all target
 layers on one stream || gather -> gamma x draft layers of draft attention on another) -> accept.  The metric is the
@@ -482,7 +482,7 @@ def run_ours(args):
 
     # per-call breakdown of one step (each call timed alone, `reps` event-bracketed repetitions)
     breakdown, other_kernels = {}, {}
-    if rank == 0:
+    if rank == 0 and not args.no_breakdown:
         st.select(cur); st.gather(cur)
         _, per = timed_reps(lambda: st.gather(cur), reps, cur, torch)
         other_kernels["gather_kv"] = {"bound": "hbm", **bandwidth_entry(st.gather_bytes(), per, 1, peaks)}
@@ -650,6 +650,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the per-call timings and whole-step times of the other configurations")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-breakdown", action="store_true",
+                    help="skip the per-call timings of the step's parts (a launch list of the run then holds whole steps only)")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

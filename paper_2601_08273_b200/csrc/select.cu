@@ -20,6 +20,8 @@
 // Section 6).  Uniform: budgets by one thread per sequence, then one CTA per frame ranks its tokens by counting.
 #include <math.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace hippo {
@@ -112,29 +114,36 @@ __global__ void __launch_bounds__(256) select_dots_kernel(const SelectParams p) 
 
 // ---- spatial score on the fp64 tensor path: one CTA per crop ---------------------------------------------------------
 // The Gram matrix of the crop's embeddings is a dense fp64 contraction over the embedding dimension: it runs on
-// mma.sync.m8n8k4.f64 (exact fp64 products of the widened inputs, fp64 accumulation; measured on B200 the instruction
-// sustains 63.7 multiply-adds per clock and SM, plain fp64 FMAs 58).  Tokens are taken in groups of eight; for the groups
-// a <= c the 8 x 8 tile G[a][c] needs one fragment per group and step of four dimensions, and for a Gram matrix the A
-// fragment of a group (row = lane / 4, dimension = lane % 4) is also its B fragment.  The embeddings are staged in shared
-// memory in their storage type, straight from global memory with cp.async (a ring of four 128-dimension chunks, no
-// registers and no conversion on the way in); warp w owns dimensions [16 w, 16 w + 16) of every chunk, and since the order
-// of a dot product's terms is free, lane l takes dimensions 4 (l % 4) .. + 3 of them: one 8-byte (bf16) load per group and
-// chunk, widened to fp64 in registers, feeds the four steps.  Every staged element is read exactly once.  The eight warps'
-// tiles are added in shared memory at the end, in a fixed order; the diagonal of G holds the squared norms.
-// A crop of 25 tokens (the paper's 5 x 5) is padded to four groups: four of the ten tiles serve its last token alone.
-// Leaving that token out of the tiles and taking its 25 dot products with plain multiply-adds (a lane per dimension and
-// partner parity) was built and measured slower (32k tokens: 506 us against 481 us for the whole selection).
-constexpr int kMmaChunk = 128;                 // dimensions per staged chunk
-constexpr int kMmaRowElems = kMmaChunk + 16;   // row stride in elements: four rows of a fragment load cover all banks once
-constexpr int kMmaStages = 4;
+// mma.sync.m8n8k4.f64 (exact fp64 products of the widened inputs, fp64 accumulation; measured on B200: one instruction per
+// 16.1 clocks and SM quarter, i.e. 63.6 multiply-adds per clock and SM, whatever the operand values and also with the
+// operands read from shared memory and widened on the way).  Tokens are taken in groups of eight; for the groups a <= c the
+// 8 x 8 tile G[a][c] needs one fragment per group and step of four dimensions, and for a Gram matrix the A fragment of a
+// group (row = lane / 4, dimension = lane % 4) is also its B fragment.  Warp w owns dimensions [16 w, 16 w + 16) of every
+// 128-dimension chunk: it stages them itself, in the storage type, straight from global memory with cp.async into a ring
+// of its own (rows back to back, so the eight rows of a fragment load are contiguous), and waits for nobody else's
+// copies: there is no block-wide barrier inside the loop.  Since the order of a dot product's terms is free, lane l takes
+// dimensions 4 (l % 4) .. + 3 of the warp's sixteen: one 8-byte (bf16) load per group and chunk, widened to fp64 in
+// registers, feeds the four steps.  Every staged element is read exactly once.  The eight warps' tiles are added in shared
+// memory at the end, in a fixed order; the diagonal of G holds the squared norms.
+// The multiply sequence is instantiated per number of groups: with the group count a run-time value every instruction of
+// it sat behind a branch of its own and the pipe was busy half of the time (32k tokens, whole selection: 472 us with the
+// branches, 351 us without, 343 us with the warps' own rings).
+// A crop of 8 n + 1 tokens (the paper's 5 x 5 = 25) would pay n + 1 tiles for its last token: that token's dot products
+// come from plain multiply-adds on the fragments the lane holds anyway (see below).
+constexpr int kMmaChunk = 128;                 // dimensions per chunk, over the eight warps
+constexpr int kMmaWarpDims = 16;               // dimensions of a chunk that one warp stages and multiplies
 constexpr int kMmaThreads = 256;
 constexpr int kMmaWarps = kMmaThreads / 32;
 constexpr int kMmaTiles = 10;                  // 4 groups: upper triangle incl. diagonal
+static_assert(kMmaWarps * kMmaWarpDims == kMmaChunk, "the warps' slices make up a chunk");
 template <typename T> struct MmaShape {
-    static constexpr int kRowBytes = kMmaRowElems * (int)sizeof(T);
-    static constexpr int kStageBytes = kMaxCrop * kRowBytes;
     static constexpr int kPiece = 16 / (int)sizeof(T);               // elements per 16-byte piece
-    static constexpr size_t kRingBytes = (size_t)kMmaStages * kStageBytes;
+    static constexpr int kPiecesPerRow = kMmaWarpDims / kPiece;
+    static constexpr int kWarpRowBytes = kMmaWarpDims * (int)sizeof(T);   // rows back to back: the eight rows of a fragment load are contiguous
+    static constexpr int kWarpStageBytes = kMaxCrop * kWarpRowBytes;
+    static constexpr int kStages = 16 / (int)sizeof(T);              // 8 chunks in flight per warp (bf16), 4 (fp32): 8 KB per warp
+    static constexpr size_t kWarpRingBytes = (size_t)kStages * kWarpStageBytes;
+    static constexpr size_t kRingBytes = (size_t)kMmaWarps * kWarpRingBytes;
     static constexpr size_t kRedBytes = (size_t)kMmaWarps * kMmaTiles * 64 * sizeof(double);
     static constexpr size_t kSmemBytes = kRingBytes > kRedBytes ? kRingBytes : kRedBytes;
 };
@@ -165,6 +174,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) select_spatial_mma_kernel(cons
     __shared__ int tok[kMaxCrop];
     __shared__ double S[kMaxCrop][kMaxCrop + 1];
     __shared__ double nrm2[kMaxCrop];
+    __shared__ double tail_red[kMmaWarps][kMaxCrop + 1];
     __shared__ int s_M;
     const int crops_per_frame = p.crops_y * p.crops_x;
     const int gframe = blockIdx.x / crops_per_frame, cr = blockIdx.x % crops_per_frame;
@@ -186,48 +196,78 @@ __global__ void __launch_bounds__(kMmaThreads, 2) select_spatial_mma_kernel(cons
     if (M == 0) return;
     const T *E = (const T *)p.embeds;
     if (M > 1) {
-        const int n_groups = (M + 7) / 8;
-        const int rows = 8 * n_groups;                       // staged rows; rows >= M are zero
-        constexpr int kPiecesPerRow = kMmaChunk / Sh::kPiece;
+        // A crop of 8n + 1 tokens (the full 5 x 5 crop: 25) would pay a whole extra group, n + 1 tiles, for its last
+        // token.  Its n * 8 dot products and its norm come from plain multiply-adds instead: at every step a lane already
+        // holds, as tile operands, token (8g + lane / 4) at the step's dimension for each group g, so all it needs besides
+        // is the last token's value at that dimension (one broadcast load per four steps), and the four lanes of a row
+        // are added at the end.
+        const bool tail = (M & 7) == 1 && M > 8;
+        const int n_groups = tail ? M / 8 : (M + 7) / 8;     // groups that go through the tiles
+        const int rows = tail ? M : 8 * n_groups;            // staged rows; rows >= M are zero
         const int n_chunks = (p.d + kMmaChunk - 1) / kMmaChunk;
+        // Each warp stages its own 16 dimensions of every chunk into a ring of its own and waits only for its own
+        // copies: no block-wide barrier inside the loop, so the warps drift apart and keep the fp64 pipe fed while
+        // others load and widen.
+        uint8_t *ring = mma_smem + (size_t)warp * Sh::kWarpRingBytes;
         auto stage_chunk = [&](int ch) {
-            uint8_t *dst = mma_smem + (size_t)(ch % kMmaStages) * Sh::kStageBytes;
-            for (int it = tid; it < rows * kPiecesPerRow; it += kMmaThreads) {
-                const int r = it / kPiecesPerRow, c = it % kPiecesPerRow;
-                const int dim = ch * kMmaChunk + c * Sh::kPiece;
+            uint8_t *dst = ring + (size_t)(ch % Sh::kStages) * Sh::kWarpStageBytes;
+            for (int it = lane; it < rows * Sh::kPiecesPerRow; it += 32) {
+                const int r = it / Sh::kPiecesPerRow, c = it % Sh::kPiecesPerRow;
+                const int dim = ch * kMmaChunk + warp * kMmaWarpDims + c * Sh::kPiece;
                 const bool live = r < M && dim < p.d;           // embed_dim is a multiple of 8: a piece is all there or not at all
-                cp_async_16(dst + r * Sh::kRowBytes + c * 16, live ? (const void *)(E + (size_t)tok[r] * p.d + dim) : (const void *)E, live ? 16 : 0);
+                cp_async_16(dst + r * Sh::kWarpRowBytes + c * 16, live ? (const void *)(E + (size_t)tok[r] * p.d + dim) : (const void *)E, live ? 16 : 0);
             }
         };
         double acc[kMmaTiles][2];
 #pragma unroll
         for (int t = 0; t < kMmaTiles; ++t) acc[t][0] = acc[t][1] = 0.0;
-        for (int s = 0; s < kMmaStages - 1; ++s) {
-            if (s < n_chunks) stage_chunk(s);
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        }
-        for (int ch = 0; ch < n_chunks; ++ch) {
-            // chunk ch has landed for every thread, and everybody is done with the slot that the next load overwrites
-            asm volatile("cp.async.wait_group %0;" ::"n"(kMmaStages - 2) : "memory");
-            __syncthreads();
-            if (ch + kMmaStages - 1 < n_chunks) stage_chunk(ch + kMmaStages - 1);
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            const T *st = reinterpret_cast<const T *>(mma_smem + (size_t)(ch % kMmaStages) * Sh::kStageBytes);
-            double frag[4][4];   // [group][step]
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                if (g < n_groups) load_frag4(st + (g * 8 + (lane >> 2)) * kMmaRowElems + warp * 16 + (lane & 3) * 4, frag[g]);
-                else frag[g][0] = frag[g][1] = frag[g][2] = frag[g][3] = 0.0;
+        double tacc[4] = {0.0, 0.0, 0.0, 0.0};               // last token x groups 0..2, and its squared norm
+        // the loop over the chunks, instantiated per (groups, tail) so that the multiply sequence is straight-line code
+        auto gram_loop = [&](auto ng_tag, auto tail_tag) {
+            constexpr int NG = decltype(ng_tag)::value;
+            constexpr bool TAIL = decltype(tail_tag)::value;
+            for (int s = 0; s < Sh::kStages - 1; ++s) {
+                if (s < n_chunks) stage_chunk(s);
+                asm volatile("cp.async.commit_group;" ::: "memory");
             }
+            for (int ch = 0; ch < n_chunks; ++ch) {
+                // this lane's copies of chunk ch have landed; after the warp barrier so have the other lanes', and every
+                // lane is done reading the slot that the next copies overwrite
+                asm volatile("cp.async.wait_group %0;" ::"n"(Sh::kStages - 2) : "memory");
+                __syncwarp();
+                if (ch + Sh::kStages - 1 < n_chunks) stage_chunk(ch + Sh::kStages - 1);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                const T *st = reinterpret_cast<const T *>(ring + (size_t)(ch % Sh::kStages) * Sh::kWarpStageBytes);
+                double frag[NG][4], tv[4] = {0.0, 0.0, 0.0, 0.0};   // [group][step]
 #pragma unroll
-            for (int step = 0; step < 4; ++step) {
-                int t = 0;
+                for (int g = 0; g < NG; ++g) load_frag4(st + (g * 8 + (lane >> 2)) * kMmaWarpDims + (lane & 3) * 4, frag[g]);
+                if (TAIL) load_frag4(st + (M - 1) * kMmaWarpDims + (lane & 3) * 4, tv);
 #pragma unroll
-                for (int ga = 0; ga < 4; ++ga)
+                for (int step = 0; step < 4; ++step) {
 #pragma unroll
-                    for (int gc = ga; gc < 4; ++gc, ++t)
-                        if (gc < n_groups) dmma_m8n8k4(acc[t][0], acc[t][1], frag[ga][step], frag[gc][step]);   // uniform over the CTA
+                    for (int ga = 0; ga < NG; ++ga)
+#pragma unroll
+                        for (int gc = ga; gc < NG; ++gc) {
+                            const int t = ga * 4 - ga * (ga - 1) / 2 + (gc - ga);   // constant after unrolling
+                            dmma_m8n8k4(acc[t][0], acc[t][1], frag[ga][step], frag[gc][step]);
+                        }
+                    if (TAIL) {
+#pragma unroll
+                        for (int g = 0; g < NG; ++g) tacc[g] = __fma_rn(frag[g][step], tv[step], tacc[g]);
+                        tacc[3] = __fma_rn(tv[step], tv[step], tacc[3]);
+                    }
+                }
             }
+        };
+        using std::integral_constant;
+        switch (n_groups * 2 + (tail ? 1 : 0)) {
+            case 2: gram_loop(integral_constant<int, 1>{}, integral_constant<bool, false>{}); break;
+            case 3: gram_loop(integral_constant<int, 1>{}, integral_constant<bool, true>{}); break;
+            case 4: gram_loop(integral_constant<int, 2>{}, integral_constant<bool, false>{}); break;
+            case 5: gram_loop(integral_constant<int, 2>{}, integral_constant<bool, true>{}); break;
+            case 6: gram_loop(integral_constant<int, 3>{}, integral_constant<bool, false>{}); break;
+            case 7: gram_loop(integral_constant<int, 3>{}, integral_constant<bool, true>{}); break;
+            default: gram_loop(integral_constant<int, 4>{}, integral_constant<bool, false>{}); break;
         }
         asm volatile("cp.async.wait_all;" ::: "memory");
         __syncthreads();
@@ -245,11 +285,30 @@ __global__ void __launch_bounds__(kMmaThreads, 2) select_spatial_mma_kernel(cons
                         mine[t * 64 + (lane >> 2) * 8 + (lane & 3) * 2 + 1] = acc[t][1];
                     }
         }
+        if (tail) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                tacc[g] += __shfl_xor_sync(0xffffffffu, tacc[g], 1);
+                tacc[g] += __shfl_xor_sync(0xffffffffu, tacc[g], 2);
+            }
+            if ((lane & 3) == 0) {
+#pragma unroll
+                for (int g = 0; g < 3; ++g)
+                    if (g < n_groups) tail_red[warp][g * 8 + (lane >> 2)] = tacc[g];
+                if (lane == 0) tail_red[warp][M - 1] = tacc[3];
+            }
+        }
         __syncthreads();
         // G[a][c] for a <= c, summed over the warps in a fixed order; then the cosines
         for (int x = tid; x < M * M; x += kMmaThreads) {
             const int a = x / M, c = x % M;
             if (a > c) continue;
+            if (tail && c == M - 1) {
+                double g = 0.0;
+                for (int w = 0; w < kMmaWarps; ++w) g += tail_red[w][a];
+                S[a][c] = g;
+                continue;
+            }
             const int ga = a >> 3, gc = c >> 3;
             const int t = ga * 4 - ga * (ga - 1) / 2 + (gc - ga);       // index of tile (ga, gc) in the upper triangle of 4 x 4
             double g = 0.0;

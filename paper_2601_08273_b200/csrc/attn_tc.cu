@@ -473,6 +473,17 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
                     locate(t, b, hk, tile);
                     const int nt = sh->tile_prefix[b + 1] - sh->tile_prefix[b];
                     const int n = (int)min((long long)(nt - tile), t_end - t);
+                    if (kMulti) {
+                        // This thread runs a few tiles ahead of the softmax threads, which fetch a segment's Q rows only when
+                        // they get there: ask for the rows now, so that they are an L2 hit by then (per query position the
+                        // G heads of a KV head are contiguous).
+                        const char *qb = (const char *)set.q[layer];
+                        for (int tq = 0; tq < p.q_len; ++tq) {
+                            const char *rows = qb + ((size_t)(b * p.q_len + tq) * p.n_q_heads + (size_t)hk * G) * (D * 2);
+                            for (int off = 0; off < G * D * 2; off += 128)
+                                asm volatile("prefetch.global.L2 [%0];" ::"l"(rows + off) : "memory");
+                        }
+                    }
                     for (int i = 0; i < n && ok; i += 2) {
                         const int pg0 = tile + i;
                         const int np = min(2, n - i);                    // the last tile of a range may hold one page
@@ -582,6 +593,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
         // Per layer: publish this CTA's partials as the softmax threads finish them, release the slot set of the next
         // layer, wait until every CTA has published the layer, merge rows blockIdx.x, blockIdx.x + gridDim.x, ...
         constexpr int V = D / 32;   // output columns per lane
+        constexpr int kMergeBatch = 24;   // partials whose loads are in flight together
         const int total_rows = B * p.q_len * p.n_q_heads;
         const size_t slot_floats = slot_float_count(R, D);
         const int Rpad = slot_rows_padded(R);
@@ -628,17 +640,24 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
                 const int n = info.y;
                 __nv_bfloat16 *o = og + (size_t)row * D + lane * V;
                 if (n == 1) continue;
-                float M = -INFINITY, L = 0.f, acc[V];
+                // All loads of a batch of kMergeBatch partials are issued before anything is used: lane j fetches the
+                // (m, l) of partial j, every lane its V output columns of all of them.  Under a saturated memory system a
+                // round trip to L2 takes microseconds, and this warp has to keep pace with the layers.
+                float M = -INFINITY, L = 0.f, acc[V];   // L: this lane's share of the weighted sums (added up below)
 #pragma unroll
                 for (int x = 0; x < V; ++x) acc[x] = 0.f;
                 const float *base = slots + (size_t)info.x * slot_floats;
-                for (int c0 = 0; c0 < n; c0 += 8) {
-                    float m[8], l[8], v[8][V];
+                for (int c0 = 0; c0 < n; c0 += kMergeBatch) {
+                    float mj = -INFINITY, lj = 0.f;
+                    if (lane < kMergeBatch && c0 + lane < n) {
+                        const float *sl = base + (size_t)(c0 + lane) * slot_floats;
+                        mj = __ldcg(sl + r);
+                        lj = __ldcg(sl + Rpad + r);
+                    }
+                    float v[kMergeBatch][V];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float *sl = base + (size_t)min(c0 + j, n - 1) * slot_floats;   // clamped; repeats are dropped below
-                        m[j] = __ldcg(sl + r);
-                        l[j] = __ldcg(sl + Rpad + r);
+                    for (int j = 0; j < kMergeBatch; ++j) {
+                        const float *sl = base + (size_t)min(c0 + j, n - 1) * slot_floats;   // clamped; repeats get weight 0
                         if (V == 4) {
                             const float4 t4 = __ldcg(reinterpret_cast<const float4 *>(sl + 2 * Rpad + (size_t)r * D + lane * V));
                             v[j][0] = t4.x; v[j][1] = t4.y; v[j][V - 2] = t4.z; v[j][V - 1] = t4.w;
@@ -647,17 +666,23 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
                             v[j][0] = t2.x; v[j][1] = t2.y;
                         }
                     }
+                    const float m_new = fmaxf(M, warp_max(mj));
+                    if (m_new == -INFINITY) continue;                       // nothing visible so far (uniform over the warp)
+                    const float f_old = (M == -INFINITY) ? 0.f : expf(M - m_new);
+                    const float w = (mj == -INFINITY) ? 0.f : expf(mj - m_new);   // 0 for lanes without a partial
+                    L = L * f_old + lj * w;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (c0 + j >= n || m[j] == -INFINITY) continue;
-                        const float m_new = fmaxf(M, m[j]);
-                        const float f_old = (M == -INFINITY) ? 0.f : expf(M - m_new), f_new = expf(m[j] - m_new);
-                        L = L * f_old + l[j] * f_new;
+                    for (int x = 0; x < V; ++x) acc[x] *= f_old;
 #pragma unroll
-                        for (int x = 0; x < V; ++x) acc[x] = acc[x] * f_old + v[j][x] * f_new;
-                        M = m_new;
+                    for (int j = 0; j < kMergeBatch; ++j) {
+                        const float wj = __shfl_sync(0xffffffffu, w, j);
+#pragma unroll
+                        for (int x = 0; x < V; ++x) acc[x] = fmaf(v[j][x], wj, acc[x]);
                     }
+                    M = m_new;
                 }
+#pragma unroll
+                for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
                 // n == 0 (a sequence shorter than q_len is skipped) leaves L = 0: its outputs are defined as zero
                 const float inv = L > 0.f ? 1.f / L : 0.f;
                 if (V == 4) {

@@ -141,7 +141,7 @@ template <typename T> struct MmaShape {
     static constexpr int kPiecesPerRow = kMmaWarpDims / kPiece;
     static constexpr int kWarpRowBytes = kMmaWarpDims * (int)sizeof(T);   // rows back to back: the eight rows of a fragment load are contiguous
     static constexpr int kWarpStageBytes = kMaxCrop * kWarpRowBytes;
-    static constexpr int kStages = 16 / (int)sizeof(T);              // 8 chunks in flight per warp (bf16), 4 (fp32): 8 KB per warp
+    static constexpr int kStages = 12 / (int)sizeof(T);              // 6 chunks in flight per warp (bf16), 3 (fp32): 6 KB per warp
     static constexpr size_t kWarpRingBytes = (size_t)kStages * kWarpStageBytes;
     static constexpr size_t kRingBytes = (size_t)kMmaWarps * kWarpRingBytes;
     static constexpr size_t kRedBytes = (size_t)kMmaWarps * kMmaTiles * 64 * sizeof(double);
@@ -168,7 +168,7 @@ __device__ __forceinline__ void load_frag4(const float *p, double *v) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kMmaThreads, 2) select_spatial_mma_kernel(const SelectParams p) {
+__global__ void __launch_bounds__(kMmaThreads, 3) select_spatial_mma_kernel(const SelectParams p) {
     using Sh = MmaShape<T>;
     extern __shared__ __align__(16) uint8_t mma_smem[];   // ring of staged chunks; reused for the warps' partial tiles
     __shared__ int tok[kMaxCrop];
@@ -209,13 +209,25 @@ __global__ void __launch_bounds__(kMmaThreads, 2) select_spatial_mma_kernel(cons
         // copies: no block-wide barrier inside the loop, so the warps drift apart and keep the fp64 pipe fed while
         // others load and widen.
         uint8_t *ring = mma_smem + (size_t)warp * Sh::kWarpRingBytes;
+        // a lane copies the same pieces (row, 16-byte column) of every chunk: source pointers and ring offsets are set up once
+        constexpr int kLanePieces = (kMaxCrop * Sh::kPiecesPerRow + 31) / 32;
+        const T *src[kLanePieces];
+        int dst_off[kLanePieces], col[kLanePieces];
+#pragma unroll
+        for (int i = 0; i < kLanePieces; ++i) {
+            const int it = lane + 32 * i;
+            const int r = it / Sh::kPiecesPerRow, c = it % Sh::kPiecesPerRow;
+            col[i] = warp * kMmaWarpDims + c * Sh::kPiece;
+            src[i] = r < M ? E + (size_t)tok[r] * p.d + col[i] : nullptr;     // rows M .. rows - 1 are zero-filled
+            dst_off[i] = it < rows * Sh::kPiecesPerRow ? r * Sh::kWarpRowBytes + c * 16 : -1;
+        }
         auto stage_chunk = [&](int ch) {
             uint8_t *dst = ring + (size_t)(ch % Sh::kStages) * Sh::kWarpStageBytes;
-            for (int it = lane; it < rows * Sh::kPiecesPerRow; it += 32) {
-                const int r = it / Sh::kPiecesPerRow, c = it % Sh::kPiecesPerRow;
-                const int dim = ch * kMmaChunk + warp * kMmaWarpDims + c * Sh::kPiece;
-                const bool live = r < M && dim < p.d;           // embed_dim is a multiple of 8: a piece is all there or not at all
-                cp_async_16(dst + r * Sh::kWarpRowBytes + c * 16, live ? (const void *)(E + (size_t)tok[r] * p.d + dim) : (const void *)E, live ? 16 : 0);
+#pragma unroll
+            for (int i = 0; i < kLanePieces; ++i) {
+                if (dst_off[i] < 0) continue;
+                const bool live = src[i] != nullptr && ch * kMmaChunk + col[i] < p.d;   // embed_dim is a multiple of 8: a piece is all there or not at all
+                cp_async_16(dst + dst_off[i], live ? (const void *)(src[i] + (size_t)ch * kMmaChunk) : (const void *)E, live ? 16 : 0);
             }
         };
         double acc[kMmaTiles][2];

@@ -66,7 +66,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;              // lazy rescale: only when a score exceeds the reference by > 2^8
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr int kLayersPerLaunch = 64;   // tensor maps and pointers of the layers travel as kernel parameters
-constexpr int kLayerRing = 3;          // slot sets for the partials of consecutive layers
+constexpr int kLayerRing = 6;          // slot sets for the partials of consecutive layers
 constexpr int kMergeWarp = kTcThreads / 32;   // the extra warp of the multi-layer kernel
 
 // Per-layer operands.  NL = 1: the single-layer calls.

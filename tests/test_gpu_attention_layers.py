@@ -93,6 +93,19 @@ def test_layers_one_unit_per_cta_and_more(hb):
         check_layers(hb, q, k, v, lens, "bf16", shuffle_seed=B)
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_layers_one_unit_with_more_contributors_than_a_merge_batch(hb, D):
+    """One (sequence, KV head) unit of 14,000 keys is split over some 30 CTAs: a row's merge takes more partials than the
+    merge warp fetches in one batch (24), so the running maximum and the rescaling across batches are exercised; values of
+    K are scaled so that the row maxima differ from partial to partial."""
+    rng = np.random.default_rng(240 + D)
+    B, q_len, Hq, Hkv = 1, 4, 4, 1
+    lens = [14000]
+    q, k, v = layer_inputs(rng, 3, B, q_len, Hq, Hkv, D, lens, "bf16")
+    k *= 4.0                                  # exact in bf16
+    check_layers(hb, q, k, v, lens, "bf16", host_lens=True)
+
+
 def test_layers_more_than_one_launch(hb):
     """70 layers: the per-layer operands travel as kernel parameters, 64 layers per launch."""
     rng = np.random.default_rng(70)

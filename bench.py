@@ -41,10 +41,10 @@ MUFU_PEAK_PER_S = 148 * 16 * 1.965e9          # 16 ex2 per clock per SM
 
 # DRAM traffic of the dominant kernel per launch (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture of
 # the workload named by the key); valid only for the kernel source it was taken on, identified by its hash.
-NCU_TRAFFIC = {"source": "paper_2601_08273_b200/csrc/attn_tc.cu", "sha1_12": "8bb61cb3b9ef",
-               # 8 layers of the same workload captured (1,086.8 MB read + 20.1 MB written), scaled by 36 / 8: traffic grows
+NCU_TRAFFIC = {"source": "paper_2601_08273_b200/csrc/attn_tc.cu", "sha1_12": "3f5bfa3f1be8",
+               # 8 layers of the same workload captured (1,084.9 MB read + 4.0 MB written), scaled by 36 / 8: traffic grows
                # in proportion to the layers
-               "bytes_per_launch": {"c2_long_video_32k": int((1086777000 + 20103424) * 36 / 8)}}
+               "bytes_per_launch": {"c2_long_video_32k": int((1084878000 + 4028928) * 36 / 8)}}
 
 
 def measured_traffic(workload):

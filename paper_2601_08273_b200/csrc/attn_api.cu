@@ -29,6 +29,7 @@ static int32_t check_shape(const char *who, int32_t batch, int32_t q_len, int32_
         return fail(HIPPO_ERR_INVALID_ARG, "%s: non-positive size", who);
     if (n_q_heads % kv->n_kv_heads) return fail(HIPPO_ERR_INVALID_ARG, "%s: n_q_heads %% n_kv_heads != 0", who);
     if ((long long)batch * kv->n_kv_heads > 16000) return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: batch*n_kv_heads > 16000", who);
+    p.kv_resident = 0;
     const int G = n_q_heads / kv->n_kv_heads, rows = q_len * G;
     if (rows > kMaxPackedRows)
         return fail(HIPPO_ERR_UNSUPPORTED_SHAPE, "%s: q_len*group = %d > %d packed rows", who, rows, kMaxPackedRows);
@@ -53,7 +54,7 @@ static int32_t check_shape(const char *who, int32_t batch, int32_t q_len, int32_
     return HIPPO_OK;
 }
 
-static int32_t attention_entry(const char *who, int32_t batch, int32_t q_len, int32_t n_q_heads,
+static int32_t attention_entry(const char *who, bool draft, int32_t batch, int32_t q_len, int32_t n_q_heads,
                                const void *q, const hippo_kv_cache_t *kv, const int32_t *kv_len,
                                const int32_t *kv_len_host, int32_t max_kv_len,
                                float softmax_scale, int32_t num_splits, void *out, float *lse, void *workspace,
@@ -67,6 +68,7 @@ static int32_t attention_entry(const char *who, int32_t batch, int32_t q_len, in
         return fail(HIPPO_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu bytes", who, workspace_bytes, L.total);
     if ((uintptr_t)workspace & 255) return fail(HIPPO_ERR_INVALID_ARG, "%s: workspace must be 256-byte aligned", who);
     p.q = q; p.out = out; p.lse = lse;
+    p.kv_resident = draft ? 1 : 0;
     p.header = (WsHeader *)workspace;
     p.counters = (int32_t *)((char *)workspace + L.counters_off);
     p.partials = (float *)((char *)workspace + L.partials_off);
@@ -100,7 +102,7 @@ int32_t hippo_verify_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, 
                                const hippo_kv_cache_t *kv, const int32_t *kv_len, const int32_t *kv_len_host,
                                int32_t max_kv_len, float softmax_scale, int32_t num_splits, void *out, float *lse,
                                void *workspace, size_t workspace_bytes, void *stream) {
-    return hippo::attention_entry("hippo_verify_attention", batch, q_len, n_q_heads, q, kv, kv_len, kv_len_host, max_kv_len,
+    return hippo::attention_entry("hippo_verify_attention", false, batch, q_len, n_q_heads, q, kv, kv_len, kv_len_host, max_kv_len,
                                   softmax_scale, num_splits, out, lse, workspace, workspace_bytes, stream);
 }
 
@@ -108,7 +110,7 @@ int32_t hippo_draft_attention(int32_t batch, int32_t q_len, int32_t n_q_heads, c
                               const hippo_kv_cache_t *kv, const int32_t *kv_len, const int32_t *kv_len_host,
                               int32_t max_kv_len, float softmax_scale, int32_t num_splits, void *out, float *lse,
                               void *workspace, size_t workspace_bytes, void *stream) {
-    return hippo::attention_entry("hippo_draft_attention", batch, q_len, n_q_heads, q, kv, kv_len, kv_len_host, max_kv_len,
+    return hippo::attention_entry("hippo_draft_attention", true, batch, q_len, n_q_heads, q, kv, kv_len, kv_len_host, max_kv_len,
                                   softmax_scale, num_splits, out, lse, workspace, workspace_bytes, stream);
 }
 
@@ -150,7 +152,7 @@ int32_t hippo_verify_attention_layers(int32_t n_layers, int32_t batch, int32_t q
         return launch_attn_tc_layers(p, n_layers, q_layers, kv_layers, out_layers, lse_layers, max_ctas, workspace, (cudaStream_t)stream);
     // shapes outside the multi-layer kernel: one single-layer call per layer, same results
     for (int l = 0; l < n_layers; ++l) {
-        int32_t rc = attention_entry(who, batch, q_len, n_q_heads, q_layers[l], &kv_layers[l], kv_len, kv_len_host, max_kv_len,
+        int32_t rc = attention_entry(who, false, batch, q_len, n_q_heads, q_layers[l], &kv_layers[l], kv_len, kv_len_host, max_kv_len,
                                      softmax_scale, 0, out_layers[l], lse_layers ? lse_layers[l] : nullptr, workspace,
                                      workspace_bytes, stream);
         if (rc != HIPPO_OK) return rc;

@@ -460,6 +460,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
             RingPos rp{0, 0};
             uint32_t issued = 0;
             bool ok = true;
+            // verification reads K and V once per call: stream them through L2; the draft's pruned cache is read again by every call
+            const uint64_t stream_pol = p.kv_resident ? l2_policy_evict_last() : l2_policy_evict_first();
             for (int layer = 0; layer < n_layers && ok; ++layer) {
                 const CUtensorMap *k_map = &set.k[layer], *v_map = &set.v[layer];
                 if (kMulti && layer + 1 < n_layers) {
@@ -500,8 +502,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
                             for (int q = 0; q < np; ++q) {
 #pragma unroll
                                 for (int c = 0; c < kChunks; ++c) {
-                                    if (kv == 0) tma_load_2d(dst + c * (2 * 8192) + q * 8192, k_map, c * 64, row[q], bar);
-                                    else tma_load_2d(dst + q * kPageBytes + c * 8192, v_map, c * 64, row[q], bar);
+                                    if (kv == 0) tma_load_2d_hint(dst + c * (2 * 8192) + q * 8192, k_map, c * 64, row[q], bar, stream_pol);
+                                    else tma_load_2d_hint(dst + q * kPageBytes + c * 8192, v_map, c * 64, row[q], bar, stream_pol);
                                 }
                             }
                         }
@@ -718,6 +720,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
         uint32_t it = 0, seg = 0;
         bool ok = true, aborted = false;
         int n_partials = 0;   // multi-layer kernel: partials this CTA has written
+        const uint64_t keep_pol = l2_policy_evict_last();
         for (int layer = 0; layer < n_layers && !aborted; ++layer) {
             const int my_cta = cta_of_layer(layer);
             long long t, t_end;
@@ -1026,7 +1029,12 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ LayerSetT<NL> set, co
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
                                     const int r = c + 4 * e4 + e;
-                                    if (store_ok && r < R) so[(size_t)r * D] = fv[e] == 0.f ? 0.f : ov[4 * e4 + e];
+                                    if (store_ok && r < R) {
+                                        // multi-layer kernel: the partial is read back by a merge warp within a few
+                                        // layers; ask L2 to keep it rather than write it out under the KV stream
+                                        if (kMulti) st_global_f32_hint(so + (size_t)r * D, fv[e] == 0.f ? 0.f : ov[4 * e4 + e], keep_pol);
+                                        else so[(size_t)r * D] = fv[e] == 0.f ? 0.f : ov[4 * e4 + e];
+                                    }
                                 }
                             }
                         }

@@ -93,6 +93,7 @@ struct AttnParams {
     int batch, q_len, n_q_heads, n_kv_heads, head_dim, group, rows;
     int n_pages, max_pages_per_seq, max_kv_len;
     int num_splits;
+    int kv_resident;             // the cache is small and read again call after call (draft): ask L2 to keep it; else it streams
     float scale;
 };
 
